@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the rank-dAD per-layer path (compress -> gather -> reconstruct) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--rank r] [--iters n]
+    python bench.py --impl reference ...       # the float64 CPU oracle on a bounded sample
+
+One step = one pass of the whole path over one synthetic batch: every linear layer of the
+configured network, all S sites per layer.  Prints ONE JSON line (rank 0).  With N > 1 ranks
+(torchrun) every rank processes its own batch of the same shape (sites and layers are
+independent: no data-path collective); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "rank-dAD compress+reconstruct layers/s"
+UNIT = "layers/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=5, help="benchmark configuration 1..5")
+    ap.add_argument("--rank", type=int, default=None, help="override the configuration's rank r")
+    ap.add_argument("--iters", type=int, default=None, help="override the power-iteration count")
+    ap.add_argument("--resident-blocks", type=int, default=4,
+                    help="distinct transformer blocks of input data kept in HBM and cycled through")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-profile-pass", action="store_true")
+    return ap.parse_args()
+
+
+def expand_layers(cfg):
+    out = []
+    for sh in cfg.layers:
+        out.extend([sh] * sh.count)
+    return out
+
+
+def workload_name(cfg, r, iters):
+    shapes = ", ".join(f"{sh.count}x {sh.h_in}->{sh.h_out}" for sh in cfg.layers)
+    return (f"config {cfg.index} ({cfg.name}): {cfg.n_layers()} linear layers = {cfg.blocks} block(s) of [{shapes}], "
+            f"S={cfg.S} sites, N={cfg.N} rows/site, {cfg.dtype} A/Delta, r={r}, iters={iters}")
+
+
+def stream_bytes_per_layer(cfg, sh, iters):
+    """Algorithmic bytes the compress passes stream for one layer: every pass reads D_s or A_s once;
+    2*iters+1 passes over each of A and D (Algorithm 2 through Eq. "reduced_iter")."""
+    e = cfg.elem_bytes
+    return {"rows_dot": ((iters + 1) * sh.h_out + iters * sh.h_in) * cfg.S * cfg.N * e,
+            "cols_acc": ((iters + 1) * sh.h_in + iters * sh.h_out) * cfg.S * cfg.N * e,
+            "rows_dot_launches": 2 * iters + 1, "cols_acc_launches": 2 * iters + 1}
+
+
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.proc = None
+        self.uuid = uuid
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+                power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def read_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg, r, iters):
+    """The oracle, as it stands, on a bounded sample: one layer of each distinct shape class (all S
+    sites), weighted by how many layers of that class a block has.  Returns (layers/s, seconds, text)."""
+    import torch
+    from oracle import dad_oracle
+    from paper_2102_09631_b200 import workloads as wl
+    shapes = list(cfg.layers)
+    # layers with the same h_in+h_out cost the same: time one per class
+    classes = {}
+    for sh in shapes:
+        classes.setdefault(sh.h_in + sh.h_out, []).append(sh)
+    total_t, parts = 0.0, []
+    per_block_t = 0.0
+    for key, members in classes.items():
+        sh = members[0]
+        A, D = wl.decaying_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, wl.seed_for(cfg.index, 0), cfg.torch_dtype)
+        Q0 = wl.start_block(cfg.S, r, sh.h_out, wl.seed_for(cfg.index, 0))
+        A64, D64, Q64 = dad_oracle.widen(A), dad_oracle.widen(D), dad_oracle.widen(Q0)
+        t0 = time.perf_counter()
+        dad_oracle.rank_dad_layer(A64, D64, Q64, iters)
+        dt = time.perf_counter() - t0
+        total_t += dt
+        count = sum(m.count for m in members)
+        per_block_t += dt * count
+        parts.append(f"{sh.h_in}->{sh.h_out} {dt:.2f}s (stands for {count}/block)")
+    layers_per_block = sum(sh.count for sh in shapes)
+    return layers_per_block / per_block_t, total_t, "one layer per shape class, all sites: " + "; ".join(parts)
+
+
+def run_reference(args):
+    from oracle import dad_oracle
+    from paper_2102_09631_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = wl.CONFIGS[args.config]
+    r = args.rank or cfg.r
+    iters = cfg.iters if args.iters is None else args.iters
+    dad_oracle.build()
+    times, sample = [], ""
+    for i in range(args.warmup + args.steps):
+        lps, secs, sample = oracle_sample(cfg, r, iters)
+        if i >= args.warmup:
+            times.append(1.0 / lps)
+    per_layer = sum(times) / len(times)
+    value = 1.0 / per_layer
+    cores = min(dad_oracle.max_threads(), cfg.S)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_layer * cfg.n_layers() * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(cfg, r, iters)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2102_09631_b200 import binding as B, build as dad_build, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    dad_build.build()
+    B.lib()
+
+    cfg = wl.CONFIGS[args.config]
+    r = args.rank or cfg.r
+    iters = cfg.iters if args.iters is None else args.iters
+    layers = expand_layers(cfg)
+    RB = max(1, min(cfg.blocks, args.resident_blocks))
+
+    # inputs: RB distinct blocks of layers resident in HBM, cycled over the network's blocks
+    data = []
+    for b in range(RB):
+        blk = []
+        for li, sh in enumerate(layers):
+            seed = wl.seed_for(cfg.index, b * len(layers) + li, rank)
+            if cfg.index == 1:
+                A, D = wl.gaussian_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+            else:
+                A, D = wl.decaying_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+            blk.append((A, D, wl.start_block(cfg.S, r, sh.h_out, seed, dev)))
+        data.append(blk)
+    plans = {}
+    for li, sh in enumerate(layers):
+        key = (sh.h_in, sh.h_out)
+        if key not in plans:
+            A, D, _ = data[0][li]
+            plans[key] = B.LayerPlan(A, D, r, iters)
+    input_bytes = sum(A.numel() * A.element_size() + D.numel() * D.element_size() for blk in data for A, D, _ in blk)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for b in range(cfg.blocks):
+            blk = data[b % RB]
+            for li, sh in enumerate(layers):
+                A, D, Q0 = blk[li]
+                plans[(sh.h_in, sh.h_out)].step(A, D, Q0, stream)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    for p in plans.values():
+        B.dad_check(p.ws)
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
+    sync_all()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    launches0 = B.dad_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    sync_all()
+    launches = B.dad_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    n_layers = cfg.n_layers()
+    value = world * n_layers / (ms_per_step * 1e-3)
+
+    # ---- per-kernel times: a second pass of the same steps with events around every launch ----
+    peaks = read_peaks()
+    roofline, kernels = None, {}
+    if not args.no_profile_pass:
+        psteps = min(args.steps, 2)
+        B.dad_timing_reset()
+        B.dad_timing_enable(True)
+        for _ in range(psteps):
+            step()
+        torch.cuda.synchronize()
+        B.dad_timing_enable(False)
+        fam = B.dad_timing_collect()
+        tot = sum(v[0] for v in fam.values()) or 1.0
+        for name, (tms, n) in sorted(fam.items(), key=lambda kv: -kv[1][0]):
+            if n:
+                kernels[name] = {"ms_per_step": tms / psteps, "launches_per_step": n / psteps, "share": tms / tot}
+        top = max(fam.items(), key=lambda kv: kv[1][0])
+        name, (tms, n) = top
+        alg = None
+        base = "rows_dot" if name.startswith("rows_dot") else "cols_acc" if name.startswith("cols_acc") else None
+        if base:
+            alg = sum(stream_bytes_per_layer(cfg, sh, iters)[base] for sh in layers) * cfg.blocks * psteps
+        if alg and n:
+            achieved = alg / (tms * 1e-3) / 1e9
+            roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                        "avg_launch_us": tms / n * 1e3, "algorithmic_bytes_per_launch": alg / n,
+                        "timing": f"CUDA events around every launch, second pass of {psteps} step(s)"}
+        else:
+            roofline = {"bound": "hbm", "kernel": name, "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": None, "traffic": None, "peak_source": peaks["source"]}
+
+    # ---- end to end: inputs start in pinned host memory, the gradient ends there ------------------
+    e2e = None
+    if not args.no_e2e:
+        host = [(A.cpu().pin_memory(), D.cpu().pin_memory(), Q0.cpu().pin_memory()) for A, D, Q0 in data[0]]
+        stage = {}
+        for li, sh in enumerate(layers):
+            key = (sh.h_in, sh.h_out)
+            if key not in stage:
+                A, D, Q0 = data[0][li]
+                stage[key] = (torch.empty_like(A), torch.empty_like(D), torch.empty_like(Q0),
+                              torch.empty(sh.h_in, sh.h_out, dtype=torch.float32).pin_memory())
+        h2d = sum(a.numel() * a.element_size() + d.numel() * d.element_size() + q.numel() * 4 for a, d, q in host) * cfg.blocks
+        d2h = sum(sh.h_in * sh.h_out * 4 for sh in layers) * cfg.blocks
+
+        def e2e_step():
+            for b in range(cfg.blocks):
+                for li, sh in enumerate(layers):
+                    key = (sh.h_in, sh.h_out)
+                    As, Ds, Qs, gh = stage[key]
+                    a, d, q = host[li]
+                    As.copy_(a, non_blocking=True)
+                    Ds.copy_(d, non_blocking=True)
+                    Qs.copy_(q, non_blocking=True)
+                    grad = plans[key].step(As, Ds, Qs, stream)
+                    gh.copy_(grad, non_blocking=True)
+
+        e2e_step()
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        sync_all()
+        ems = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ems], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        e2e = {"value": world * n_layers * args.e2e_steps / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import dad_oracle
+        dad_oracle.build()
+        lps, secs, sample = oracle_sample(cfg, r, iters)
+        cpu = {"value": lps, "unit": UNIT, "cores": min(dad_oracle.max_threads(), cfg.S), "kind": "oracle",
+               "sample": sample, "seconds": secs}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "bf16", "data": "synthetic",
+                "config": {"workload": workload_name(cfg, r, iters),
+                           "l2": f"inputs larger than L2: {RB} resident block(s), {input_bytes / 1e9:.2f} GB, cycled",
+                           "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+                "kernels": kernels,
+                "stream_gbs": sum(sum(v for k, v in stream_bytes_per_layer(cfg, sh, iters).items() if not k.endswith("launches"))
+                                  for sh in layers) * cfg.blocks / (ms_per_step * 1e-3) / 1e9}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

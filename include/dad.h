@@ -1,0 +1,191 @@
+/*
+ * dad.h -- C ABI of libdad: the per-layer hot path of distributed auto-differentiation
+ * (dAD) and its rank-reduced form (rank-dAD), as hand-written CUDA for sm_100a.
+ *
+ * For one linear layer, every site s of S holds its input activations A_s (N x h_in) and
+ * the back-propagated errors D_s (N x h_out, the paper's Delta_i).  The site gradient is
+ * the product A_s^T D_s (Eq. "local_grad", Sec. 3.1).  dAD ships A_s and D_s and multiplies
+ * the concatenated batch (Sec. 3.2); rank-dAD first reduces them to rank-r factors with
+ * structured power iterations on the implicit product (Algorithm 2, Sec. 3.3.1), stacks the
+ * factors of all sites and reconstructs the gradient from the stacks (Algorithm 1).
+ * Sites are slices of one device buffer; nothing here communicates between GPUs.
+ *
+ * Conventions
+ *   - Every matrix is dense row-major.  "DEVICE" pointers are CUDA device memory of the
+ *     current device, owned by the caller, who keeps them alive until the work queued on
+ *     `cuda_stream` has finished.  "HOST" pointers are ordinary host memory, read or written
+ *     before the call returns.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *     only enqueue work; none of them synchronises, allocates device memory or keeps state
+ *     between calls (exceptions are stated at the entry point).
+ *   - Inputs are never written.  Outputs are overwritten, never accumulated into.
+ *   - Every call returns a dad_status.  Errors the host can see (NULL pointers, bad shapes,
+ *     ranks, strides, alignment, a workspace that is too small) are returned before anything
+ *     is launched.  On error the outputs are unspecified but no write leaves the buffers.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with
+ *     DAD_ERR_CUDA.
+ */
+#ifndef DAD_H_
+#define DAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DAD_OK = 0,
+  DAD_ERR_NULL = 1,      /* a required pointer is NULL                                        */
+  DAD_ERR_SHAPE = 2,     /* S, N, h_in, h_out, K, iters or a stride is out of range           */
+  DAD_ERR_DTYPE = 3,     /* dtype is neither DAD_F32 nor DAD_BF16                             */
+  DAD_ERR_RANK = 4,      /* r < 1, r > DAD_MAX_RANK or r > min(h_in, h_out)                   */
+  DAD_ERR_WORKSPACE = 5, /* ws is smaller than dad_workspace_bytes() says                     */
+  DAD_ERR_ALIGN = 6,     /* a pointer or stride misses the alignment stated below             */
+  DAD_ERR_CUDA = 7,      /* the CUDA runtime reported an error (no device, bad launch, ...)   */
+  DAD_ERR_TIMEOUT = 8,   /* a bounded device-side wait ran out (reported by dad_check)        */
+  DAD_ERR_NUMERIC = 9    /* a NaN/Inf reached the orthonormalisation (reported by dad_check)  */
+} dad_status;
+
+typedef enum { DAD_F32 = 0, DAD_BF16 = 1 } dad_dtype;
+
+#define DAD_MAX_RANK 64
+
+/*
+ * One linear layer seen from all S sites.
+ *   A: element (s, n, a) at A[s*strideA + n*ldA + a],  0<=n<N, 0<=a<h_in
+ *   D: element (s, n, b) at D[s*strideD + n*ldD + b],  0<=b<h_out
+ * Strides are in ELEMENTS of `dtype`.  ldA >= h_in, ldD >= h_out; strideA >= N*ldA (when S>1),
+ * likewise strideD.  A and D base pointers must be aligned to 16 bytes; for DAD_BF16 the
+ * tensor-core kernels are used when, in addition, h_in, h_out, ldA, ldD, strideA and strideD
+ * are multiples of 8 elements (16 bytes) -- any other layout takes the slower general kernels,
+ * with the same results.  Factors, gradients and start blocks are always fp32, contiguous.
+ */
+typedef struct {
+  int32_t S;            /* number of sites (>= 1)                         */
+  int64_t N;            /* rows per site (batch x tokens), >= 1            */
+  int64_t h_in, h_out;  /* layer width in / out, >= 1                      */
+  dad_dtype dtype;      /* storage type of A and D                        */
+  int64_t ldA, ldD;     /* row strides in elements                        */
+  int64_t strideA, strideD; /* site strides in elements                   */
+} dad_layer;
+
+/*
+ * Bytes a site transmits for this layer (host arithmetic, exact, no device work):
+ *   dad_bytes_dad : N*(h_in+h_out)*e, both component matrices at their storage width e
+ *                   (Sec. 3.1, "m+n against m*n"; Sec. 3.2)
+ *   dad_bytes_rank: r*(h_in+h_out)*4, the two rank-r fp32 factors (Sec. 2, the
+ *                   Theta(r(h_i+h_{i+1})) bandwidth of rank methods; Sec. 3.3)
+ *   dad_bytes_dsgd: h_in*h_out*4, the full fp32 gradient that dSGD ships (Sec. 1)
+ * A NULL or invalid layer gives 0.
+ */
+uint64_t dad_bytes_dad(const dad_layer* layer);
+uint64_t dad_bytes_rank(const dad_layer* layer, int r);
+uint64_t dad_bytes_dsgd(const dad_layer* layer);
+
+/*
+ * Scratch bytes dad_rank_compress / dad_full_grad need for this layer (the larger of the two;
+ * 0 if the arguments are invalid).  The caller allocates at least this much DEVICE memory,
+ * aligned to 256 bytes, and may reuse it for any later call with the same or smaller needs.
+ * Two calls that overlap in time on the GPU must not share a workspace.
+ */
+size_t dad_workspace_bytes(const dad_layer* layer, int r, int iters);
+
+/*
+ * Uncompressed dAD gradient (Sec. 3.2; Eq. "local_grad"; Sec. 5.1): the product of the
+ * batch-concatenated component matrices,
+ *     grad[a][b] = sum_s sum_n A_s[n][a] * D_s[n][b],
+ * which equals the gradient of the pooled batch exactly (up to rounding order).
+ *   A, D     DEVICE, as laid out by `layer`
+ *   grad     DEVICE, h_in x h_out fp32, contiguous, 16-byte aligned
+ *   bytes_tx HOST, S entries, or NULL: entry s receives dad_bytes_dad(layer)
+ *   ws       DEVICE scratch of ws_bytes >= dad_workspace_bytes(layer, 1, 0)
+ * DAD_F32 inputs are multiplied in fp32 (FMA); DAD_BF16 inputs on the tensor cores with fp32
+ * accumulation.
+ */
+dad_status dad_full_grad(const dad_layer* layer, const void* A, const void* D, float* grad,
+                         uint64_t* bytes_tx, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Structured power iterations, all r vectors of a site advanced together (Algorithm 2;
+ * Eq. "nabla_iter" evaluated through A and D as in Eq. "reduced_iter", never forming the
+ * h_in x h_out gradient; the peel term of Eq. "peel" realised as orthonormalisation of the
+ * r vectors).  Independently for every site s:
+ *     G <- Q0_s
+ *     repeat iters times:  G <- orth( D_s^T ( A_s ( A_s^T ( D_s G^T ))) )     (rows of G)
+ *     Q_s = G,  P_s = ( A_s^T ( D_s G^T ) )^T,  sigma_s[j] = || P_s[j] ||
+ * so that P_s^T Q_s is the projection of A_s^T D_s on the span of the r directions found.
+ * orth = thin QR with positive diagonal; a vector whose remainder after projection is below
+ * 1e-12 (DAD_F32) or 1e-6 (DAD_BF16) of its length is set to exactly zero.
+ *   r        1 <= r <= min(h_in, h_out, DAD_MAX_RANK);  iters >= 0
+ *   Q0       DEVICE, S x r x h_out fp32: the start vectors g_0 ~ N(0,1), supplied by the caller
+ *   P        DEVICE, S x r x h_in  fp32 (out)
+ *   Q        DEVICE, S x r x h_out fp32 (out; may alias Q0)
+ *   sigma    DEVICE, S x r fp32 (out) or NULL
+ *   ws       DEVICE scratch of ws_bytes >= dad_workspace_bytes(layer, r, iters)
+ * DAD_F32: all products accumulate in fp64 and intermediates are kept in fp64.
+ * DAD_BF16: fp32 accumulation; the fp32 factor operand of each product enters as a
+ * two-term bf16 split, so products carry about 16 significant bits of the factor.
+ */
+dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* D, int r, int iters,
+                             const float* Q0, float* P, float* Q, float* sigma,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Gather at the aggregator (Algorithm 1, the two vertcat lines): site s's factors become rows
+ * s*r .. s*r+r-1 of the stacks, and each site is charged what it sent.
+ *   P, Q       DEVICE, S x r x h_in and S x r x h_out fp32 (as written by dad_rank_compress)
+ *   Pcat, Qcat DEVICE, (S*r) x h_in and (S*r) x h_out fp32 (out).  Pcat == P and Qcat == Q are
+ *              allowed: the stacks then are the factor buffers themselves and nothing is copied.
+ *   bytes_tx   HOST, S entries, or NULL: entry s receives dad_bytes_rank(layer, r)
+ * Only S, h_in and h_out of `layer` are read.
+ */
+dad_status dad_gather_factors(const dad_layer* layer, int r, const float* P, const float* Q,
+                              float* Pcat, float* Qcat, uint64_t* bytes_tx, void* cuda_stream);
+
+/*
+ * Reconstruction (Algorithm 1, the P^T Q step): the sum over the K = S*r stacked rows of the
+ * outer products of the factors,
+ *     grad[a][b] = sum_k Pcat[k][a] * Qcat[k][b].
+ *   Pcat, Qcat DEVICE, K x h_in and K x h_out fp32, contiguous, 16-byte aligned
+ *   grad       DEVICE, h_in x h_out fp32 (out)
+ *   math       DAD_F32: fp32 FMA.  DAD_BF16: tensor cores, factors rounded to bf16, fp32
+ *              accumulation (for layers whose inputs were bf16 already).
+ *   ws         DEVICE scratch of ws_bytes >= dad_reconstruct_workspace_bytes(h_in, h_out, K),
+ *              may be NULL when that is 0
+ */
+size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math);
+dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat,
+                           float* grad, dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Device-side status of the work that used `ws`: synchronises `cuda_stream`, reads the status
+ * word at the head of the workspace and returns it (DAD_OK, DAD_ERR_TIMEOUT, DAD_ERR_NUMERIC),
+ * or DAD_ERR_CUDA if the stream reports an error.  This is the only call that synchronises.
+ */
+dad_status dad_check(const void* ws, void* cuda_stream);
+
+/* Kernels launched by this library in this process so far (all threads); for accounting. */
+uint64_t dad_launch_count(void);
+
+const char* dad_status_string(dad_status status);
+
+/*
+ * Instrumentation for benchmarks (the paper has no counterpart).  While enabled, every kernel this
+ * library launches is bracketed by CUDA events on its own stream, which costs a little time per
+ * launch; dad_timing_collect() waits for the recorded events (it synchronises) and adds the elapsed
+ * time of each launch to the total of its kernel family, returning the number of families seen.
+ * dad_timing_name/ms/launches read family i; dad_timing_reset() clears the totals.
+ */
+void dad_timing_enable(int on);
+int dad_timing_collect(void);
+void dad_timing_reset(void);
+const char* dad_timing_name(int i);
+double dad_timing_ms(int i);
+uint64_t dad_timing_launches(int i);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAD_H_ */

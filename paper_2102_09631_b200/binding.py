@@ -1,0 +1,235 @@
+"""Thin Python binding of libdad (include/dad.h): same names, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams only); every
+step of the path runs in the library's own kernels.  There is no fallback: if libdad.so is
+missing or cannot be loaded, or a call returns an error status, a RuntimeError is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdad.so")
+
+DAD_OK = 0
+DAD_F32, DAD_BF16 = 0, 1
+DAD_MAX_RANK = 64
+STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD_ERR_RANK", "DAD_ERR_WORKSPACE",
+                "DAD_ERR_ALIGN", "DAD_ERR_CUDA", "DAD_ERR_TIMEOUT", "DAD_ERR_NUMERIC"]
+
+# every symbol include/dad.h declares
+EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
+           "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
+           "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
+           "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
+
+
+class dad_layer(ctypes.Structure):
+    _fields_ = [("S", ctypes.c_int32), ("N", ctypes.c_int64), ("h_in", ctypes.c_int64), ("h_out", ctypes.c_int64),
+                ("dtype", ctypes.c_int), ("ldA", ctypes.c_int64), ("ldD", ctypes.c_int64),
+                ("strideA", ctypes.c_int64), ("strideD", ctypes.c_int64)]
+
+
+class DadError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name} ({lib().dad_status_string(status).decode()})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libdad.so (built in-tree by paper_2102_09631_b200.build); fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2102_09631_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, u64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint64)
+        lp = ctypes.POINTER(dad_layer)
+        L.dad_bytes_dad.argtypes = [lp]
+        L.dad_bytes_dad.restype = ctypes.c_uint64
+        L.dad_bytes_rank.argtypes = [lp, ctypes.c_int]
+        L.dad_bytes_rank.restype = ctypes.c_uint64
+        L.dad_bytes_dsgd.argtypes = [lp]
+        L.dad_bytes_dsgd.restype = ctypes.c_uint64
+        L.dad_workspace_bytes.argtypes = [lp, ctypes.c_int, ctypes.c_int]
+        L.dad_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_full_grad.argtypes = [lp, vp, vp, vp, u64p, vp, ctypes.c_size_t, vp]
+        L.dad_full_grad.restype = ctypes.c_int
+        L.dad_rank_compress.argtypes = [lp, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.dad_rank_compress.restype = ctypes.c_int
+        L.dad_gather_factors.argtypes = [lp, ctypes.c_int, vp, vp, vp, vp, u64p, vp]
+        L.dad_gather_factors.restype = ctypes.c_int
+        L.dad_reconstruct_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int]
+        L.dad_reconstruct_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_reconstruct.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, ctypes.c_int, vp,
+                                      ctypes.c_size_t, vp]
+        L.dad_reconstruct.restype = ctypes.c_int
+        L.dad_check.argtypes = [vp, vp]
+        L.dad_check.restype = ctypes.c_int
+        L.dad_launch_count.argtypes = []
+        L.dad_launch_count.restype = ctypes.c_uint64
+        L.dad_status_string.argtypes = [ctypes.c_int]
+        L.dad_status_string.restype = ctypes.c_char_p
+        L.dad_timing_enable.argtypes = [ctypes.c_int]
+        L.dad_timing_enable.restype = None
+        L.dad_timing_collect.restype = ctypes.c_int
+        L.dad_timing_reset.restype = None
+        L.dad_timing_name.argtypes = [ctypes.c_int]
+        L.dad_timing_name.restype = ctypes.c_char_p
+        L.dad_timing_ms.argtypes = [ctypes.c_int]
+        L.dad_timing_ms.restype = ctypes.c_double
+        L.dad_timing_launches.argtypes = [ctypes.c_int]
+        L.dad_timing_launches.restype = ctypes.c_uint64
+        _lib = L
+    return _lib
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return DAD_F32
+    if t == torch.bfloat16:
+        return DAD_BF16
+    raise TypeError(f"A and D must be float32 or bfloat16, got {t}")
+
+
+def make_layer(A: torch.Tensor, D: torch.Tensor) -> dad_layer:
+    """Descriptor of a layer whose sites are the leading dimension: A is S x N x h_in, D is S x N x h_out
+    (innermost dimension contiguous; row and site strides are taken from the tensors)."""
+    if A.dim() != 3 or D.dim() != 3 or A.shape[:2] != D.shape[:2] or A.dtype != D.dtype:
+        raise ValueError("A must be S x N x h_in and D S x N x h_out of one dtype")
+    if A.stride(2) != 1 or D.stride(2) != 1:
+        raise ValueError("innermost dimension must be contiguous")
+    S, N, h_in = A.shape
+    return dad_layer(S, N, h_in, D.shape[2], _dtype_code(A.dtype), A.stride(1), D.stride(1), A.stride(0), D.stride(0))
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else ctypes.c_void_p(0)
+
+
+def _check(status: int, where: str):
+    if status != DAD_OK:
+        raise DadError(status, where)
+
+
+def dad_bytes_dad(layer: dad_layer) -> int:
+    return int(lib().dad_bytes_dad(ctypes.byref(layer)))
+
+
+def dad_bytes_rank(layer: dad_layer, r: int) -> int:
+    return int(lib().dad_bytes_rank(ctypes.byref(layer), r))
+
+
+def dad_bytes_dsgd(layer: dad_layer) -> int:
+    return int(lib().dad_bytes_dsgd(ctypes.byref(layer)))
+
+
+def dad_workspace_bytes(layer: dad_layer, r: int, iters: int) -> int:
+    return int(lib().dad_workspace_bytes(ctypes.byref(layer), r, iters))
+
+
+def dad_launch_count() -> int:
+    return int(lib().dad_launch_count())
+
+
+def new_workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def dad_full_grad(layer: dad_layer, A, D, grad, bytes_tx=None, ws=None, stream=None):
+    """grad (h_in x h_out fp32) <- sum_s A_s^T D_s; bytes_tx: optional ctypes uint64 array of S entries."""
+    st = lib().dad_full_grad(ctypes.byref(layer), _ptr(A), _ptr(D), _ptr(grad), bytes_tx, _ptr(ws),
+                             ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_full_grad")
+
+
+def dad_rank_compress(layer: dad_layer, A, D, r: int, iters: int, Q0, P, Q, sigma, ws, stream=None):
+    st = lib().dad_rank_compress(ctypes.byref(layer), _ptr(A), _ptr(D), r, iters, _ptr(Q0), _ptr(P), _ptr(Q),
+                                 _ptr(sigma), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_rank_compress")
+
+
+def dad_gather_factors(layer: dad_layer, r: int, P, Q, Pcat, Qcat, bytes_tx=None, stream=None):
+    st = lib().dad_gather_factors(ctypes.byref(layer), r, _ptr(P), _ptr(Q), _ptr(Pcat), _ptr(Qcat), bytes_tx,
+                                  _stream(stream))
+    _check(st, "dad_gather_factors")
+
+
+def dad_reconstruct_workspace_bytes(h_in: int, h_out: int, K: int, math: int) -> int:
+    return int(lib().dad_reconstruct_workspace_bytes(h_in, h_out, K, math))
+
+
+def dad_reconstruct(h_in: int, h_out: int, K: int, Pcat, Qcat, grad, math: int = DAD_F32, ws=None, stream=None):
+    st = lib().dad_reconstruct(h_in, h_out, K, _ptr(Pcat), _ptr(Qcat), _ptr(grad), math, _ptr(ws),
+                               ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_reconstruct")
+
+
+def dad_check(ws, stream=None):
+    _check(lib().dad_check(_ptr(ws), _stream(stream)), "dad_check")
+
+
+def dad_timing_enable(on: bool):
+    lib().dad_timing_enable(1 if on else 0)
+
+
+def dad_timing_reset():
+    lib().dad_timing_reset()
+
+
+def dad_timing_collect() -> dict:
+    """{kernel family: (total ms, launches)} of the launches timed since the last reset (synchronises)."""
+    n = lib().dad_timing_collect()
+    return {lib().dad_timing_name(i).decode(): (float(lib().dad_timing_ms(i)), int(lib().dad_timing_launches(i)))
+            for i in range(n)}
+
+
+def bytes_array(S: int):
+    return (ctypes.c_uint64 * S)()
+
+
+class LayerPlan:
+    """Buffers for one layer shape, allocated once: factors, stacks, gradient and workspace.
+    `step` runs compress -> gather -> reconstruct on the current stream (marshalling only)."""
+
+    def __init__(self, A: torch.Tensor, D: torch.Tensor, r: int, iters: int, zero_copy_gather: bool = False):
+        self.layer = make_layer(A, D)
+        L = self.layer
+        dev = A.device
+        self.r, self.iters = r, iters
+        self.P = torch.empty(L.S, r, L.h_in, device=dev, dtype=torch.float32)
+        self.Q = torch.empty(L.S, r, L.h_out, device=dev, dtype=torch.float32)
+        self.sigma = torch.empty(L.S, r, device=dev, dtype=torch.float32)
+        if zero_copy_gather:
+            self.Pcat, self.Qcat = self.P.view(L.S * r, L.h_in), self.Q.view(L.S * r, L.h_out)
+        else:
+            self.Pcat = torch.empty(L.S * r, L.h_in, device=dev, dtype=torch.float32)
+            self.Qcat = torch.empty(L.S * r, L.h_out, device=dev, dtype=torch.float32)
+        self.grad = torch.empty(L.h_in, L.h_out, device=dev, dtype=torch.float32)
+        self.math = L.dtype
+        nws = dad_workspace_bytes(L, r, iters)
+        if nws == 0:
+            raise ValueError("invalid layer / rank / iteration count")
+        self.ws = new_workspace(max(nws, dad_reconstruct_workspace_bytes(L.h_in, L.h_out, L.S * r, self.math)), dev)
+        self.bytes_tx = bytes_array(L.S)
+
+    def step(self, A, D, Q0, stream=None):
+        L = self.layer
+        dad_rank_compress(L, A, D, self.r, self.iters, Q0, self.P, self.Q, self.sigma, self.ws, stream)
+        dad_gather_factors(L, self.r, self.P, self.Q, self.Pcat, self.Qcat, self.bytes_tx, stream)
+        dad_reconstruct(L.h_in, L.h_out, L.S * self.r, self.Pcat, self.Qcat, self.grad, self.math, self.ws, stream)
+        return self.grad

@@ -1,0 +1,100 @@
+// Shared declarations of the libdad translation units: launch accounting, the workspace
+// layout of dad_rank_compress, and the host-side launchers of every kernel family.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "dad.h"
+
+namespace dad {
+
+extern std::atomic<uint64_t> g_launches;
+
+// Optional per-kernel timing (dad_timing_*): CUDA events recorded around every launch on the
+// launching stream, summed per tag when collected.  Off by default; no cost when off.
+extern std::atomic<bool> g_timing;
+void timing_mark(const char* tag, cudaStream_t st, bool begin);
+
+// Launch a kernel under a tag, count it and fold its launch error into `err` (first error wins).
+#define DAD_LAUNCH(err, tag, kernel, grid, block, smem, stream, ...)            \
+  do {                                                                          \
+    const bool t__ = ::dad::g_timing.load(std::memory_order_relaxed);           \
+    if (t__) ::dad::timing_mark(tag, stream, true);                             \
+    kernel<<<grid, block, smem, stream>>>(__VA_ARGS__);                         \
+    cudaError_t e__ = cudaGetLastError();                                       \
+    if (t__) ::dad::timing_mark(tag, stream, false);                            \
+    ::dad::g_launches.fetch_add(1, std::memory_order_relaxed);                  \
+    if ((err) == cudaSuccess) (err) = e__;                                      \
+  } while (0)
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// ---- geometry shared by launchers and the workspace carve --------------------------------
+constexpr int kColsAccThreads = 128;  // columns per CTA of the column-slab product
+constexpr int kGramChunk = 64;        // columns per CTA of the Gram kernel
+
+// Row splits of the column-slab product Z = Y^T X, chosen from the shape alone so that the
+// launch fills the GPU; identical for workspace sizing and launching.
+int cols_acc_splits(int S, int64_t N, int64_t h);
+
+// Workspace of dad_rank_compress; all offsets in bytes from the (256-aligned) base.
+struct CompressWs {
+  size_t status;        // int32 status word (+ padding)
+  size_t counters;      // uint32 arrival counters of the split reductions
+  size_t n_counters;
+  size_t G;             // S*r*h_out accumulator-type iterate (fp64 pipeline only)
+  size_t Y;             // S*N*r
+  size_t Z;             // S*r*h_in
+  size_t partial;       // S*splits*r*max(h) partial column slabs
+  size_t gram_partial;  // S*chunks*r*r doubles
+  size_t gram;          // S*r*r doubles (Cholesky factor after the Gram kernel)
+  size_t tratio;        // S*r doubles: R_jj / ||column|| after the first pass
+  size_t dead;          // S*r bytes
+  // tensor-core pipeline: bf16 two-term splits of the small operands
+  size_t Fsplit;        // S*2*rp*max(h) bf16: split of the r x h factor operand (hi plane, lo plane)
+  size_t Ysplit;        // S*2*rp*Npad bf16: split of the N x r operand, stored transposed (rp x Npad)
+  size_t total;
+};
+CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64);
+
+// ---- launchers (all asynchronous on `st`; return the first CUDA error) ------------------------
+// Y[s][n][j] = sum_c X[s][n][c] * F[s][j][c]      X: N x h (ld, site stride), F: r x h, Y: N x r
+template <typename TAcc>
+cudaError_t rows_dot(dad_dtype dt, const void* X, int64_t ld, int64_t stride, int S, int64_t N, int64_t h,
+                     const TAcc* F, int r, TAcc* Y, cudaStream_t st);
+
+// Z[s][j][c] = sum_n Y[s][n][j] * X[s][n][c]      Z: r x h; also written as fp32 to out32 if given
+template <typename TAcc>
+cudaError_t cols_acc(dad_dtype dt, const void* X, int64_t ld, int64_t stride, int S, int64_t N, int64_t h,
+                     const TAcc* Y, int r, TAcc* Z, float* out32, TAcc* partial, unsigned* counters,
+                     cudaStream_t st);
+
+// One Cholesky-QR pass on the rows of G (S x r x h, in place): Gram -> factor -> triangular solve.
+// pass = 0: first pass (records R_jj/||g_j||); pass = 1: second pass, zeroes rows whose total
+// remainder is <= tol of their length.  out32 (optional) receives an fp32 copy of the result.
+template <typename T>
+cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, double* gram_partial,
+                        double* gram, double* tratio, unsigned char* dead, unsigned* counters,
+                        int* status, float* out32, cudaStream_t st);
+
+// C[a][b] = sum_{s,n} X[s][n][a] * Y[s][n][b]  (fp32 FMA), C: hx x hy fp32 contiguous
+cudaError_t gemm_tn_simt(dad_dtype dt, const void* X, int64_t ldX, int64_t strideX, const void* Y,
+                         int64_t ldY, int64_t strideY, int S, int64_t N, int64_t hx, int64_t hy, float* C,
+                         cudaStream_t st);
+
+cudaError_t copy_two(const float* a, float* a_out, size_t na, const float* b, float* b_out, size_t nb,
+                     cudaStream_t st);
+cudaError_t widen_f32_to_f64(const float* in, double* out, size_t n, cudaStream_t st);
+template <typename T>
+cudaError_t row_norms(const T* M, int64_t rows, int64_t h, float* out, cudaStream_t st);
+
+}  // namespace dad

@@ -1,0 +1,148 @@
+// General fp32-FMA kernel for the two dense products of the path, both of the form
+//   C[a][b] = sum_k X[k][a] * Y[k][b]
+// with the contraction index k as the row index of both operands:
+//   - the uncompressed dAD gradient sum_s A_s^T D_s (Sec. 3.2; k runs over all sites' rows),
+//   - the reconstruction Pcat^T Qcat (Algorithm 1; k runs over the S*r stacked factor rows).
+// Used for fp32 inputs (where bf16 tensor-core products would miss the 1e-5 parity bound) and
+// for layouts the tensor-core kernel does not take.  Also small helpers: factor gather copy,
+// fp32 -> fp64 widening, row norms.
+#include "common.cuh"
+
+namespace dad {
+
+constexpr int BM = 64, BN = 64, BK = 16;
+
+template <typename TIn>
+__global__ void __launch_bounds__(256)
+gemm_tn_kernel(const TIn* __restrict__ X, int64_t ldX, int64_t strideX, const TIn* __restrict__ Y, int64_t ldY,
+               int64_t strideY, int64_t N, int64_t Ktot, int64_t hx, int64_t hy, float* __restrict__ C) {
+  __shared__ __align__(16) float Xs[BK][BM];
+  __shared__ __align__(16) float Ys[BK][BN];
+  const int tid = threadIdx.x;
+  const int tx = tid % 16, ty = tid / 16;
+  const int64_t a0 = (int64_t)blockIdx.y * BM, b0 = (int64_t)blockIdx.x * BN;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  for (int64_t k0 = 0; k0 < Ktot; k0 += BK) {
+#pragma unroll
+    for (int i = 0; i < (BK * BM) / 256; ++i) {
+      const int idx = tid + i * 256;
+      const int kk = idx / BM, col = idx % BM;
+      const int64_t k = k0 + kk;
+      float xv = 0.f, yv = 0.f;
+      if (k < Ktot) {
+        const int64_t s = k / N, n = k % N;
+        if (a0 + col < hx) xv = to_float(X[s * strideX + n * ldX + a0 + col]);
+        if (b0 + col < hy) yv = to_float(Y[s * strideY + n * ldY + b0 + col]);
+      }
+      Xs[kk][col] = xv;
+      Ys[kk][col] = yv;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 xa = *reinterpret_cast<const float4*>(&Xs[kk][ty * 4]);
+      const float4 yb = *reinterpret_cast<const float4*>(&Ys[kk][tx * 4]);
+      const float xr[4] = {xa.x, xa.y, xa.z, xa.w};
+      const float yr[4] = {yb.x, yb.y, yb.z, yb.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xr[i], yr[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t a = a0 + ty * 4 + i;
+    if (a >= hx) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t b = b0 + tx * 4 + j;
+      if (b < hy) C[a * hy + b] = acc[i][j];
+    }
+  }
+}
+
+cudaError_t gemm_tn_simt(dad_dtype dt, const void* X, int64_t ldX, int64_t strideX, const void* Y,
+                         int64_t ldY, int64_t strideY, int S, int64_t N, int64_t hx, int64_t hy, float* C,
+                         cudaStream_t st) {
+  dim3 grid((unsigned)ceil_div(hy, BN), (unsigned)ceil_div(hx, BM));
+  cudaError_t err = cudaSuccess;
+  const int64_t Ktot = (int64_t)S * N;
+  if (dt == DAD_F32)
+    DAD_LAUNCH(err, "gemm_tn_simt", (gemm_tn_kernel<float>), grid, 256, 0, st, (const float*)X, ldX, strideX, (const float*)Y, ldY,
+               strideY, N, Ktot, hx, hy, C);
+  else
+    DAD_LAUNCH(err, "gemm_tn_simt", (gemm_tn_kernel<__nv_bfloat16>), grid, 256, 0, st, (const __nv_bfloat16*)X, ldX, strideX,
+               (const __nv_bfloat16*)Y, ldY, strideY, N, Ktot, hx, hy, C);
+  return err;
+}
+
+// ---- small helpers ---------------------------------------------------------------------------
+__global__ void copy_two_kernel(const float* __restrict__ a, float* __restrict__ a_out, size_t na,
+                                const float* __restrict__ b, float* __restrict__ b_out, size_t nb) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < na + nb; i += stride) {
+    if (i < na) {
+      if (a_out != a) a_out[i] = a[i];
+    } else {
+      if (b_out != b) b_out[i - na] = b[i - na];
+    }
+  }
+}
+
+cudaError_t copy_two(const float* a, float* a_out, size_t na, const float* b, float* b_out, size_t nb,
+                     cudaStream_t st) {
+  cudaError_t err = cudaSuccess;
+  size_t blocks = (na + nb + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  DAD_LAUNCH(err, "gather_copy", copy_two_kernel, (unsigned)blocks, 256, 0, st, a, a_out, na, b, b_out, nb);
+  return err;
+}
+
+__global__ void widen_kernel(const float* __restrict__ in, double* __restrict__ out, size_t n) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = (double)in[i];
+}
+
+cudaError_t widen_f32_to_f64(const float* in, double* out, size_t n, cudaStream_t st) {
+  cudaError_t err = cudaSuccess;
+  size_t blocks = (n + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  DAD_LAUNCH(err, "widen", widen_kernel, (unsigned)blocks, 256, 0, st, in, out, n);
+  return err;
+}
+
+// out[row] = || M[row] ||_2, one warp per row (sigma_j = ||P_j||, Algorithm 2's sqrt(v^T C v)).
+template <typename T>
+__global__ void __launch_bounds__(256) row_norms_kernel(const T* __restrict__ M, int64_t rows, int64_t h,
+                                                        float* __restrict__ out) {
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  double acc = 0.0;
+  for (int64_t c = lane; c < h; c += 32) {
+    const double v = (double)M[row * h + c];
+    acc += v * v;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) out[row] = (float)sqrt(acc);
+}
+
+template <typename T>
+cudaError_t row_norms(const T* M, int64_t rows, int64_t h, float* out, cudaStream_t st) {
+  cudaError_t err = cudaSuccess;
+  DAD_LAUNCH(err, "row_norms", (row_norms_kernel<T>), (unsigned)ceil_div(rows, 8), 256, 0, st, M, rows, h, out);
+  return err;
+}
+template cudaError_t row_norms<float>(const float*, int64_t, int64_t, float*, cudaStream_t);
+template cudaError_t row_norms<double>(const double*, int64_t, int64_t, float*, cudaStream_t);
+
+}  // namespace dad

@@ -1,0 +1,169 @@
+// Orthonormalisation of the r iterate vectors of a site (the block form of the deflation of
+// Eq. "peel": each vector loses its components along the ones before it), as Cholesky-QR:
+//   Gram = G G^T (fp64, r x r)  ->  Gram = L L^T  ->  rows of G <- L^{-1} G.
+// This is the thin QR with positive diagonal (R = L^T).  One pass leaves an orthogonality
+// defect of about 1e-16 * cond(G)^2, so the pass is applied twice.  Pivots are kept from
+// collapsing: a pivot below (1e-7)^2 of the vector's squared length is raised to that value in
+// the first pass (the vector then comes out short instead of wrong), and the second pass, which
+// sees a well-conditioned matrix, decides from the product of both passes' diagonals whether the
+// vector carried any new direction; if not it is set to exactly zero.
+#include "common.cuh"
+
+namespace dad {
+
+constexpr double kPivotFloor = 1e-14;  // (1e-7)^2, relative to the squared length of the vector
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int pass, double tol,
+                     double* __restrict__ partial, double* __restrict__ Lout, double* __restrict__ tratio,
+                     unsigned char* __restrict__ dead, unsigned* __restrict__ counters, int* __restrict__ status) {
+  extern __shared__ double sm[];  // max(r * (kGramChunk + 1), r * (r + 1)) doubles
+  const int s = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
+  const T* Gs = G + (int64_t)s * r * h;
+  const int64_t c0 = (int64_t)chunk * kGramChunk;
+  constexpr int LD = kGramChunk + 1;
+  for (int idx = tid; idx < r * kGramChunk; idx += 256) {
+    const int j = idx / kGramChunk, cc = idx % kGramChunk;
+    sm[j * LD + cc] = (c0 + cc < h) ? (double)Gs[(int64_t)j * h + c0 + cc] : 0.0;
+  }
+  __syncthreads();
+  double* mine = partial + ((int64_t)s * chunks + chunk) * r * r;
+  for (int p = tid; p < r * r; p += 256) {
+    const int i = p / r, j = p % r;
+    if (j <= i) {
+      double acc = 0.0;
+#pragma unroll 8
+      for (int cc = 0; cc < kGramChunk; ++cc) acc += sm[i * LD + cc] * sm[j * LD + cc];
+      mine[p] = acc;
+    }
+  }
+  __shared__ bool is_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned old = atomicAdd(counters + s, 1u);
+    is_last = (old == (unsigned)chunks - 1u);
+    if (is_last) counters[s] = 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // Sum the chunk partials in chunk order, then factor in shared memory.
+  const int LR = r + 1;
+  const double* src = partial + (int64_t)s * chunks * r * r;
+  for (int p = tid; p < r * r; p += 256) {
+    const int i = p / r, j = p % r;
+    if (j <= i) {
+      double v = 0.0;
+      for (int q = 0; q < chunks; ++q) v += __ldcg(src + (int64_t)q * r * r + p);
+      sm[i * LR + j] = v;
+    }
+  }
+  __shared__ double ljj;
+  __shared__ int col_dead;
+  __syncthreads();
+  double* Ls = Lout + (int64_t)s * r * r;
+  for (int j = 0; j < r; ++j) {
+    if (tid == 0) {
+      // the squared length of vector j before projection is its Gram diagonal: kept in tratio/dead bookkeeping
+      const double d = sm[j * LR + j];
+      // original diagonal = d + sum_l L_jl^2
+      double orig = d;
+      for (int l = 0; l < j; ++l) orig += sm[j * LR + l] * sm[j * LR + l];
+      int is_dead = 0;
+      double piv = d;
+      if (!(orig == orig) || orig > 1.7e308) {
+        *status = (int)DAD_ERR_NUMERIC;
+        is_dead = 1;
+      } else if (!(orig > 0.0)) {
+        is_dead = 1;
+      } else {
+        const double floor_ = kPivotFloor * orig;
+        if (!(piv > floor_)) piv = floor_;
+      }
+      double l = is_dead ? 1.0 : sqrt(piv);
+      if (!is_dead) {
+        if (pass == 0) {
+          tratio[(int64_t)s * r + j] = l / sqrt(orig);
+        } else {
+          // total remainder relative to the vector's length before the first pass
+          const double total = tratio[(int64_t)s * r + j] * l;
+          if (!(total > tol)) is_dead = 1;
+        }
+      } else if (pass == 0) {
+        tratio[(int64_t)s * r + j] = 0.0;
+      }
+      ljj = l;
+      col_dead = is_dead;
+      dead[(int64_t)s * r + j] = (unsigned char)is_dead;
+      sm[j * LR + j] = l;
+    }
+    __syncthreads();
+    const double l = ljj;
+    const int dd = col_dead;
+    for (int i = j + 1 + tid; i < r; i += 256) sm[i * LR + j] = dd ? 0.0 : sm[i * LR + j] / l;
+    __syncthreads();
+    const int m = r - j - 1;  // trailing block rows j+1..r-1
+    for (int p = tid; p < m * m; p += 256) {
+      const int i = j + 1 + p / m, k = j + 1 + p % m;
+      if (k <= i) sm[i * LR + k] -= sm[i * LR + j] * sm[k * LR + j];
+    }
+    __syncthreads();
+  }
+  for (int p = tid; p < r * r; p += 256) {
+    const int i = p / r, j = p % r;
+    Ls[p] = (j <= i) ? sm[i * LR + j] : 0.0;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128)
+tri_solve_kernel(T* __restrict__ G, int r, int64_t h, const double* __restrict__ L,
+                 const unsigned char* __restrict__ dead, float* __restrict__ out32) {
+  extern __shared__ double sm[];  // r*r (L) + r*128 (solved column values)
+  double* Ls = sm;
+  double* qs = sm + r * r;
+  const int s = blockIdx.y, tid = threadIdx.x;
+  for (int p = tid; p < r * r; p += 128) Ls[p] = L[(int64_t)s * r * r + p];
+  __syncthreads();
+  const int64_t b = (int64_t)blockIdx.x * 128 + tid;
+  if (b >= h) return;
+  T* Gs = G + (int64_t)s * r * h;
+  const unsigned char* ds = dead + (int64_t)s * r;
+  for (int j = 0; j < r; ++j) {
+    double v = (double)Gs[(int64_t)j * h + b];
+    for (int l = 0; l < j; ++l) v -= Ls[j * r + l] * qs[l * 128 + tid];
+    v = ds[j] ? 0.0 : v / Ls[j * r + j];
+    qs[j * 128 + tid] = v;
+    Gs[(int64_t)j * h + b] = (T)v;
+    if (out32) out32[((int64_t)s * r + j) * h + b] = (float)v;
+  }
+}
+
+template <typename T>
+cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, double* gram_partial,
+                        double* gram, double* tratio, unsigned char* dead, unsigned* counters,
+                        int* status, float* out32, cudaStream_t st) {
+  cudaError_t err = cudaSuccess;
+  const int chunks = (int)ceil_div(h, kGramChunk);
+  const int a = r * (kGramChunk + 1), b = r * (r + 1);
+  const size_t smem1 = sizeof(double) * (size_t)(a > b ? a : b);
+  const size_t smem2 = sizeof(double) * (size_t)(r * r + r * 128);
+  // the opt-in is per device and cheap, so it is simply made on every call
+  if (smem2 > 48 * 1024) {
+    err = cudaFuncSetAttribute(tri_solve_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    if (err != cudaSuccess) return err;
+  }
+  DAD_LAUNCH(err, "gram_cholesky", (gram_cholesky_kernel<T>), dim3((unsigned)chunks, (unsigned)S), 256, smem1, st, G, r, h, chunks, pass,
+             tol, gram_partial, gram, tratio, dead, counters, status);
+  DAD_LAUNCH(err, "tri_solve", (tri_solve_kernel<T>), dim3((unsigned)ceil_div(h, 128), (unsigned)S), 128, smem2, st, G, r, h, gram,
+             dead, out32);
+  return err;
+}
+template cudaError_t cholqr_pass<float>(float*, int, int, int64_t, int, double, double*, double*, double*,
+                                        unsigned char*, unsigned*, int*, float*, cudaStream_t);
+template cudaError_t cholqr_pass<double>(double*, int, int, int64_t, int, double, double*, double*, double*,
+                                         unsigned char*, unsigned*, int*, float*, cudaStream_t);
+
+}  // namespace dad

@@ -1,0 +1,250 @@
+"""Parity of the CUDA path (through the C ABI) with the float64 CPU oracle on the same seeded inputs.
+
+Bars (relative Frobenius error): 1e-5 for fp32 inputs, 2e-2 for bf16 inputs with fp32 accumulation;
+transmitted byte counts are bit-exact.  Any orthonormal basis of the subspace found gives the same
+P_s^T Q_s, so parity is asserted on P_s^T Q_s, on the reconstructed gradient and on Q Q^T = I;
+the raw factors are compared as well where the spectrum separates the vectors.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2102_09631_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL = {torch.float32: 1e-5, torch.bfloat16: 2e-2}
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2102_09631_b200 import build, binding
+    assert torch.cuda.is_available(), "these tests need the B200"
+    build.build()
+    binding.lib()
+    return binding
+
+
+def rel(x, ref):
+    x = np.asarray(x, dtype=np.float64)
+    return float(np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def run_gpu_layer(B, A, D, Q0, r, iters, math=None):
+    """compress -> gather -> reconstruct and full_grad on the GPU; returns host float64 arrays."""
+    dev = torch.device("cuda:0")
+    Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
+    plan = B.LayerPlan(Ad, Dd, r, iters)
+    if math is not None:
+        plan.math = math
+    plan.step(Ad, Dd, Q0d)
+    full = torch.empty_like(plan.grad)
+    tx_dad = B.bytes_array(plan.layer.S)
+    B.dad_full_grad(plan.layer, Ad, Dd, full, tx_dad, plan.ws)
+    B.dad_check(plan.ws)
+    torch.cuda.synchronize()
+    f = lambda t: t.double().cpu().numpy()
+    return dict(P=f(plan.P), Q=f(plan.Q), sigma=f(plan.sigma), Pcat=f(plan.Pcat), Qcat=f(plan.Qcat), grad=f(plan.grad),
+                full=f(full), tx_rank=list(plan.bytes_tx), tx_dad=list(tx_dad), layer=plan.layer)
+
+
+def check_layer(oracle, B, A, D, Q0, r, iters, tol, ortho_tol=1e-4, compare_factors=False):
+    S, N, h_in = A.shape
+    h_out = D.shape[2]
+    g = run_gpu_layer(B, A, D, Q0, r, iters)
+    o = oracle.rank_dad_layer(A, D, Q0, iters)
+    e = A.element_size()
+    # bytes: bit-exact
+    assert g["tx_rank"] == [int(x) for x in o["bytes_tx"]] == [oracle.bytes_rank(r, h_in, h_out)] * S
+    assert g["tx_dad"] == [oracle.bytes_dad(N, h_in, h_out, e)] * S
+    # uncompressed dAD gradient
+    assert rel(g["full"], oracle.full_grad(A, D)) <= tol
+    # per-site projected gradients, orthonormality, sigma
+    for s in range(S):
+        ref = o["P"][s].T @ o["Q"][s]
+        got = g["P"][s].T @ g["Q"][s]
+        assert rel(got, ref) <= tol, (s, rel(got, ref))
+        live = [j for j in range(r) if np.any(g["Q"][s][j] != 0.0)]
+        live_o = [j for j in range(r) if np.any(o["Q"][s][j] != 0.0)]
+        assert len(live) == len(live_o)
+        Ql = g["Q"][s][live]
+        if iters > 0:  # with no iteration Q is the caller's start block, returned as it came
+            assert np.linalg.norm(Ql @ Ql.T - np.eye(len(live))) <= ortho_tol
+        assert np.allclose(g["sigma"][s], np.linalg.norm(g["P"][s], axis=1), rtol=1e-5, atol=1e-30)
+        if compare_factors:
+            assert rel(g["Q"][s], o["Q"][s]) <= 50 * tol and rel(g["P"][s], o["P"][s]) <= 50 * tol
+    # gather: stacks are the factors in site order, bit for bit
+    assert np.array_equal(g["Pcat"], g["P"].reshape(S * r, h_in))
+    assert np.array_equal(g["Qcat"], g["Q"].reshape(S * r, h_out))
+    # reconstruction
+    assert rel(g["grad"], o["grad"]) <= tol, rel(g["grad"], o["grad"])
+    return g, o
+
+
+def test_config1_single_linear_layer(oracle, B):
+    cfg = wl.CONFIGS[1]
+    A, D, Q0 = wl.layer_inputs(cfg, cfg.layers[0], 0)
+    g, o = check_layer(oracle, B, A, D, Q0, cfg.r, cfg.iters, TOL[torch.float32])
+    # "compare to full A^T D": the rank-4 estimate of a flat-spectrum gradient is far from it, equally
+    # so for both implementations (an approximation error, not a parity criterion)
+    err_gpu = rel(g["grad"], g["full"])
+    err_ref = rel(o["grad"], oracle.full_grad(A, D))
+    assert abs(err_gpu - err_ref) < 1e-5 and 0.3 < err_ref < 1.0
+
+
+def test_config2_mlp_all_layers(oracle, B):
+    cfg = wl.CONFIGS[2]
+    mb = wl.mlp_layers(S=cfg.S, N=cfg.N)
+    for i, shape in enumerate(cfg.layers):
+        A, D = mb.A[i].float(), mb.D[i].float()
+        assert A.shape == (cfg.S, cfg.N, shape.h_in) and D.shape == (cfg.S, cfg.N, shape.h_out)
+        Q0 = wl.start_block(cfg.S, cfg.r, shape.h_out, wl.seed_for(2, i))
+        check_layer(oracle, B, A, D, Q0, cfg.r, cfg.iters, TOL[torch.float32])
+
+
+def test_config3_encoder_layer_projections(oracle, B):
+    cfg = wl.CONFIGS[3]
+    layers = wl.encoder_layers(S=cfg.S)
+    seen = set()
+    for i, (name, A, D) in enumerate(layers):
+        if (A.shape[2], D.shape[2]) in seen and name != "o":
+            continue  # q, k, v share a shape and an input; one of them and the output projection suffice
+        seen.add((A.shape[2], D.shape[2]))
+        assert A.dtype == torch.bfloat16 and A.shape[1] == cfg.N
+        Q0 = wl.start_block(cfg.S, cfg.r, D.shape[2], wl.seed_for(3, i))
+        check_layer(oracle, B, A, D, Q0, cfg.r, cfg.iters, TOL[torch.bfloat16], ortho_tol=1e-3)
+
+
+@pytest.mark.parametrize("N,h_in,h_out,r,iters,dtype", [
+    (6304 // 8, 768, 3072, 16, 3, torch.bfloat16),   # ViT-B ffn_up shape, ragged row count (788 = 6*128 + 20)
+    (300, 1024, 1024, 4, 1, torch.bfloat16),          # GPT-2-medium attention projection, smallest sweep point
+    (515, 4096, 1024, 64, 1, torch.bfloat16),         # ffn_down at the largest rank, odd row count
+    (257, 200, 136, 10, 2, torch.bfloat16),           # widths that are multiples of 8 but of no tile
+    (100, 70, 50, 7, 2, torch.bfloat16),              # widths that are not multiples of 8: general kernels
+    (130, 96, 40, 5, 3, torch.float32),
+])
+def test_shape_slices(oracle, B, N, h_in, h_out, r, iters, dtype):
+    S = 2
+    seed = 4242 + N + h_in
+    A, D = wl.decaying_layer(S, N, h_in, h_out, seed, dtype)
+    Q0 = wl.start_block(S, r, h_out, seed)
+    check_layer(oracle, B, A, D, Q0, r, iters, TOL[dtype], ortho_tol=1e-3 if dtype == torch.bfloat16 else 1e-4)
+
+
+def test_factors_match_on_separated_spectrum(oracle, B):
+    """With well separated singular values and enough iterations each vector is determined up to
+    rounding (thin QR with positive diagonal fixes the sign), so the raw factors agree too."""
+    S, N, h_in, h_out, r = 2, 64, 48, 40, 3
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 99, torch.float32, modes=6, noise=0.0)
+    Q0 = wl.start_block(S, r, h_out, 99)
+    check_layer(oracle, B, A, D, Q0, r, 12, 1e-5, compare_factors=True)
+
+
+def test_rank_exceeding_true_rank_is_exact(oracle, B):
+    """r >= rank(A_s^T D_s): the estimate reproduces the uncompressed gradient, surplus vectors are zero."""
+    S, N, h_in, h_out, r = 3, 5, 64, 48, 8   # batch of 5 rows: rank <= 5 < r
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 7)
+    Q0 = wl.start_block(S, r, h_out, 7)
+    g, o = check_layer(oracle, B, A, D, Q0, r, 1, 1e-5)
+    assert rel(g["grad"], g["full"]) <= 1e-5
+    for s in range(S):
+        assert sum(1 for j in range(r) if np.all(g["Q"][s][j] == 0.0)) == r - N
+        assert np.all(g["sigma"][s][N:] == 0.0)
+
+
+def test_edge_shapes(oracle, B):
+    # one row, one site, r = 1; r = min(h); zero iterations; strided (non-contiguous) rows and sites
+    A, D = wl.gaussian_layer(1, 1, 8, 8, 1)
+    check_layer(oracle, B, A, D, wl.start_block(1, 1, 8, 1), 1, 2, 1e-5)
+    A, D = wl.gaussian_layer(2, 40, 16, 6, 2)
+    check_layer(oracle, B, A, D, wl.start_block(2, 6, 6, 2), 6, 2, 1e-5)
+    check_layer(oracle, B, A, D, wl.start_block(2, 3, 6, 3), 3, 0, 1e-5)
+    Abig, Dbig = wl.gaussian_layer(3, 50, 40, 24, 3)
+    A, D = Abig[:, :33, :32], Dbig[:, :33, :16]   # views: ld > h, site stride > N*ld
+    assert not A.is_contiguous()
+    dev = torch.device("cuda:0")
+    Ad, Dd = Abig.to(dev)[:, :33, :32], Dbig.to(dev)[:, :33, :16]
+    Q0 = wl.start_block(3, 4, 16, 4)
+    plan = B.LayerPlan(Ad, Dd, 4, 2)
+    assert plan.layer.ldA == 40 and plan.layer.strideA == 50 * 40
+    plan.step(Ad, Dd, Q0.to(dev))
+    B.dad_check(plan.ws)
+    o = oracle.rank_dad_layer(A.contiguous(), D.contiguous(), Q0, 2)
+    assert rel(plan.grad.double().cpu().numpy(), o["grad"]) <= 1e-5
+
+
+def test_zero_copy_gather_and_determinism(oracle, B):
+    dev = torch.device("cuda:0")
+    A, D = wl.decaying_layer(4, 700, 256, 512, 11, torch.bfloat16)
+    Q0 = wl.start_block(4, 16, 512, 11)
+    Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
+    outs = []
+    for zero_copy in (False, True, True):
+        plan = B.LayerPlan(Ad, Dd, 16, 2, zero_copy_gather=zero_copy)
+        plan.step(Ad, Dd, Q0d)
+        B.dad_check(plan.ws)
+        outs.append((plan.grad.clone(), plan.P.clone(), plan.Q.clone()))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)          # aliasing the stacks changes nothing
+    for a, b in zip(outs[1], outs[2]):
+        assert torch.equal(a, b)          # two runs agree bit for bit
+
+
+def test_nan_input_is_reported_not_trapped(B):
+    dev = torch.device("cuda:0")
+    A, D = wl.gaussian_layer(1, 32, 16, 16, 5)
+    D[0, 3, 2] = float("nan")
+    plan = B.LayerPlan(A.to(dev), D.to(dev), 4, 1)
+    plan.step(A.to(dev), D.to(dev), wl.start_block(1, 4, 16, 5).to(dev))
+    with pytest.raises(B.DadError, match="NUMERIC"):
+        B.dad_check(plan.ws)
+    # the context is intact: a clean call afterwards succeeds
+    A, D = wl.gaussian_layer(1, 32, 16, 16, 6)
+    plan = B.LayerPlan(A.to(dev), D.to(dev), 4, 1)
+    plan.step(A.to(dev), D.to(dev), wl.start_block(1, 4, 16, 6).to(dev))
+    B.dad_check(plan.ws)
+
+
+def test_reconstruct_and_full_grad_at_full_size_on_sampled_rows(oracle, B):
+    """Largest shapes of the GPT-2-medium configuration; the oracle computes sampled output rows."""
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(31)
+    h_in, h_out, K = 1024, 4096, 1024
+    Pcat = torch.randn(K, h_in, generator=g)
+    Qcat = torch.randn(K, h_out, generator=g)
+    rows = [0, 1, 63, 64, 517, 1023]
+    for math in (B.DAD_F32, B.DAD_BF16):
+        grad = torch.empty(h_in, h_out, device=dev)
+        ws = B.new_workspace(B.dad_reconstruct_workspace_bytes(h_in, h_out, K, math), dev)
+        B.dad_reconstruct(h_in, h_out, K, Pcat.to(dev), Qcat.to(dev), grad, math, ws)
+        ref = oracle.reconstruct(Pcat[:, rows], Qcat)
+        assert rel(grad[rows].double().cpu().numpy(), ref) <= (1e-5 if math == B.DAD_F32 else 2e-2)
+    S, N = 16, 4096
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 32, torch.bfloat16, device=dev)
+    L = B.make_layer(A, D)
+    grad = torch.empty(h_in, h_out, device=dev)
+    ws = B.new_workspace(B.dad_workspace_bytes(L, 1, 0), dev)
+    B.dad_full_grad(L, A, D, grad, None, ws)
+    torch.cuda.synchronize()
+    ref = oracle.full_grad(A[:, :, rows].cpu(), D.cpu())
+    assert rel(grad[rows].double().cpu().numpy(), ref) <= 2e-2
+
+
+def test_compress_at_full_size_on_sampled_sites(oracle, B):
+    """GPT-2-medium ffn_up layer exactly as the benchmark launches it (S=16, N=4096, r=16, 3 iterations);
+    sites are independent, so the oracle recomputes two of them from the same inputs."""
+    dev = torch.device("cuda:0")
+    cfg = wl.CONFIGS[5]
+    shape = cfg.layers[1]
+    A, D, Q0 = wl.layer_inputs(cfg, shape, 1, device=dev)
+    plan = B.LayerPlan(A, D, cfg.r, cfg.iters)
+    plan.step(A, D, Q0)
+    B.dad_check(plan.ws)
+    sites = [0, 11]
+    Po, Qo, _ = oracle.spi_block(A[sites].cpu(), D[sites].cpu(), Q0[sites].cpu(), cfg.iters)
+    for i, s in enumerate(sites):
+        got = plan.P[s].double().cpu().numpy().T @ plan.Q[s].double().cpu().numpy()
+        assert rel(got, Po[i].T @ Qo[i]) <= 2e-2
+        Qg = plan.Q[s].double().cpu().numpy()
+        assert np.linalg.norm(Qg @ Qg.T - np.eye(cfg.r)) <= 1e-3
+    assert list(plan.bytes_tx) == [oracle.bytes_rank(cfg.r, shape.h_in, shape.h_out)] * cfg.S
