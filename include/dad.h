@@ -88,7 +88,9 @@ uint64_t dad_bytes_dsgd(const dad_layer* layer);
  * Scratch bytes dad_rank_compress / dad_full_grad need for this layer (the larger of the two;
  * 0 if the arguments are invalid).  The caller allocates at least this much DEVICE memory,
  * aligned to 256 bytes, and may reuse it for any later call with the same or smaller needs.
- * Two calls that overlap in time on the GPU must not share a workspace.
+ * Two calls that overlap in time on the GPU must not share a workspace.  The first 256 bytes
+ * hold the status words dad_check() reads: they must be zero when the workspace is first handed
+ * to the library (one cudaMemset); afterwards the library maintains them.
  */
 size_t dad_workspace_bytes(const dad_layer* layer, int r, int iters);
 
@@ -161,8 +163,10 @@ dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* 
 
 /*
  * Device-side status of the work that used `ws`: synchronises `cuda_stream`, reads the status
- * word at the head of the workspace and returns it (DAD_OK, DAD_ERR_TIMEOUT, DAD_ERR_NUMERIC),
- * or DAD_ERR_CUDA if the stream reports an error.  This is the only call that synchronises.
+ * words at the head of the workspace -- one written by the last dad_rank_compress on it, one by
+ * the last dad_full_grad / dad_reconstruct on it -- and returns the first that is not DAD_OK
+ * (DAD_ERR_TIMEOUT, DAD_ERR_NUMERIC), or DAD_ERR_CUDA if the stream reports an error.  Each of
+ * those calls clears its own word when it starts.  This is the only call that synchronises.
  */
 dad_status dad_check(const void* ws, void* cuda_stream);
 

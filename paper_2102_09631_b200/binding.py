@@ -147,7 +147,9 @@ def dad_launch_count() -> int:
 
 
 def new_workspace(nbytes: int, device) -> torch.Tensor:
-    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    ws[:256].zero_()  # the status words must start out clear
+    return ws
 
 
 def dad_full_grad(layer: dad_layer, A, D, grad, bytes_tx=None, ws=None, stream=None):

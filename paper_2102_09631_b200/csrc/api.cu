@@ -13,6 +13,7 @@ static bool layer_ok(const dad_layer* L) {
   if (!L) return false;
   if (L->S < 1 || L->N < 1 || L->h_in < 1 || L->h_out < 1) return false;
   if (L->S > 65535) return false;
+  if (L->N > 0x7fffffff || L->h_in > 0x7fffffff || L->h_out > 0x7fffffff) return false;
   return true;
 }
 
@@ -22,15 +23,22 @@ static dad_status validate_layer(const dad_layer* L) {
   if (!layer_ok(L)) return DAD_ERR_SHAPE;
   if (L->ldA < L->h_in || L->ldD < L->h_out) return DAD_ERR_SHAPE;
   if (L->S > 1 && (L->strideA < L->N * L->ldA || L->strideD < L->N * L->ldD)) return DAD_ERR_SHAPE;
-  // 63-bit element counts
-  const double big = 9.0e18;
+  const double big = 9.0e18;  // element counts must fit 63 bits
   if ((double)L->S * (double)L->N * (double)(L->ldA > L->ldD ? L->ldA : L->ldD) * 8.0 > big) return DAD_ERR_SHAPE;
   return DAD_OK;
 }
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64) {
+bool tc_eligible(const dad_layer& L) {
+  if (L.dtype != DAD_BF16) return false;
+  if ((L.h_in | L.h_out | L.ldA | L.ldD) % 8 != 0) return false;
+  if (L.S > 1 && ((L.strideA | L.strideD) % 8 != 0)) return false;
+  if ((double)L.strideA * 2.0 >= 1.0e12 || (double)L.strideD * 2.0 >= 1.0e12) return false;  // TMA strides < 2^40 bytes
+  return tmap_encoder_available();
+}
+
+CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc) {
   CompressWs w;
   memset(&w, 0, sizeof(w));
   const size_t acc = f64 ? 8 : 4;
@@ -45,13 +53,15 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64) {
   w.G = off;
   off = align_up(off + (f64 ? S * rr * ho * acc : 0), 256);
   w.Y = off;
-  off = align_up(off + S * N * rr * acc, 256);
+  off = align_up(off + (tc ? 0 : S * N * rr * acc), 256);
   w.Z = off;
-  off = align_up(off + S * rr * hi * acc, 256);
-  const int s_in = cols_acc_splits(L.S, L.N, L.h_in), s_out = cols_acc_splits(L.S, L.N, L.h_out);
+  off = align_up(off + (tc ? 0 : S * rr * hi * acc), 256);
   size_t part = 0;
-  if (s_in > 1) part = S * (size_t)s_in * rr * hi * acc;
-  if (s_out > 1 && S * (size_t)s_out * rr * ho * acc > part) part = S * (size_t)s_out * rr * ho * acc;
+  if (!tc) {
+    const int s_in = cols_acc_splits(L.S, L.N, L.h_in), s_out = cols_acc_splits(L.S, L.N, L.h_out);
+    if (s_in > 1) part = S * (size_t)s_in * rr * hi * acc;
+    if (s_out > 1 && S * (size_t)s_out * rr * ho * acc > part) part = S * (size_t)s_out * rr * ho * acc;
+  }
   w.partial = off;
   off = align_up(off + part, 256);
   w.gram_partial = off;
@@ -62,12 +72,57 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64) {
   off = align_up(off + S * rr * 8, 256);
   w.dead = off;
   off = align_up(off + S * rr, 256);
-  w.Fsplit = off;
-  w.Ysplit = off;
+  w.Fq = w.Fz = w.Yt = w.tc_partial = off;
+  if (tc) {
+    const size_t rp = (size_t)umma_rank_pad(r);
+    w.Npad = (int64_t)align_up(N, 8);
+    w.Fq = off;
+    off = align_up(off + S * 2 * rp * ho * 2, 256);
+    w.Fz = off;
+    off = align_up(off + S * 2 * rp * hi * 2, 256);
+    w.Yt = off;
+    off = align_up(off + S * 2 * rp * (size_t)w.Npad * 2, 256);
+    const size_t p_in = (size_t)umma_cols_acc_splits(L.S, L.N, L.h_in) * (size_t)ceil_div(L.h_in, 128);
+    const size_t p_out = (size_t)umma_cols_acc_splits(L.S, L.N, L.h_out) * (size_t)ceil_div(L.h_out, 128);
+    w.tc_partial = off;
+    off = align_up(off + S * (p_in > p_out ? p_in : p_out) * 128 * rp * 4, 256);
+  }
   w.total = off;
   return w;
 }
 
+GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands) {
+  GemmWs w;
+  memset(&w, 0, sizeof(w));
+  size_t off = 0;
+  w.status = off;
+  off += 256;
+  const size_t tiles = (size_t)(ceil_div(hx, 128) * ceil_div(hy, 128));
+  const int splits = umma_gemm_splits(hx, hy, ceil_div(N, 64) * S);
+  w.n_counters = tiles;
+  w.counters = off;
+  off = align_up(off + tiles * sizeof(unsigned), 256);
+  w.partial = off;
+  off = align_up(off + (splits > 1 ? tiles * (size_t)splits * 128 * 128 * 4 : 0), 256);
+  w.Xb = w.Yb = off;
+  if (convert_operands) {
+    w.Xb = off;
+    off = align_up(off + (size_t)S * N * hx * 2, 256);
+    w.Yb = off;
+    off = align_up(off + (size_t)S * N * hy * 2, 256);
+  }
+  w.total = off;
+  return w;
+}
+
+#define DAD_STEP(call)                  \
+  do {                                  \
+    err = (call);                       \
+    if (err != cudaSuccess) return err; \
+  } while (0)
+
+// General pipeline: fp32 inputs with fp64 accumulation (TAcc = double), or bf16 inputs in a layout
+// the tensor-core kernels do not take, with fp32 accumulation (TAcc = float).
 template <typename TAcc>
 static cudaError_t run_compress(const dad_layer& L, const void* A, const void* D, int r, int iters, const float* Q0,
                                 float* P, float* Q, float* sigma, char* ws, const CompressWs& w, cudaStream_t st) {
@@ -98,26 +153,90 @@ static cudaError_t run_compress(const dad_layer& L, const void* A, const void* D
     if (Q != Q0) err = cudaMemcpyAsync(Q, Q0, sizeof(float) * (size_t)S * r * ho, cudaMemcpyDeviceToDevice, st);
   }
   if (err != cudaSuccess) return err;
-#define DAD_STEP(call)          \
-  do {                          \
-    err = (call);               \
-    if (err != cudaSuccess) return err; \
-  } while (0)
   for (int k = 0; k < iters; ++k) {
-    DAD_STEP(rows_dot<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, G, r, Y, st));                        // Y = D G^T
+    DAD_STEP(rows_dot<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, G, r, Y, st));                           // Y = D G^T
     DAD_STEP(cols_acc<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Y, r, Z, nullptr, part, ctr_cols, st));  // Z = Y^T A
-    DAD_STEP(rows_dot<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Z, r, Y, st));                        // W = A Z^T
+    DAD_STEP(rows_dot<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Z, r, Y, st));                           // W = A Z^T
     DAD_STEP(cols_acc<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, Y, r, G, nullptr, part, ctr_cols, st));  // Gt = W^T D
-    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr, st));
+    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr,
+                               nullptr, 0, st));
     float* q32 = (f64 && k == iters - 1) ? Q : nullptr;
-    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, ctr_gram, status, q32, st));
+    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, ctr_gram, status, q32, nullptr,
+                               0, st));
   }
   DAD_STEP(rows_dot<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, G, r, Y, st));
   DAD_STEP(cols_acc<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Y, r, Z, P, part, ctr_cols, st));
   if (sigma) DAD_STEP(row_norms<TAcc>(Z, (int64_t)S * r, hi, sigma, st));
-#undef DAD_STEP
   return cudaSuccess;
 }
+
+// Tensor-core pipeline for bf16 inputs: every product runs as tcgen05 MMAs with fp32 accumulation;
+// the small fp32 operand of each product (G, Y, Z, W) is handed on as two bf16 planes (hi + lo).
+static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void* D, int r, int iters, const float* Q0,
+                                   float* P, float* Q, float* sigma, char* ws, const CompressWs& w, cudaStream_t st) {
+  const int S = L.S;
+  const int64_t N = L.N, hi = L.h_in, ho = L.h_out;
+  const int rp = umma_rank_pad(r);
+  cudaError_t err = cudaMemsetAsync(ws + w.status, 0, w.counters + w.n_counters * sizeof(unsigned) - w.status, st);
+  if (err != cudaSuccess) return err;
+  int* status = reinterpret_cast<int*>(ws + w.status);
+  unsigned* ctr_cols = reinterpret_cast<unsigned*>(ws + w.counters);
+  unsigned* ctr_gram = ctr_cols + (w.n_counters - (size_t)S);
+  double* gram_partial = reinterpret_cast<double*>(ws + w.gram_partial);
+  double* gram = reinterpret_cast<double*>(ws + w.gram);
+  double* tratio = reinterpret_cast<double*>(ws + w.tratio);
+  unsigned char* dead = reinterpret_cast<unsigned char*>(ws + w.dead);
+  __nv_bfloat16* Fq = reinterpret_cast<__nv_bfloat16*>(ws + w.Fq);
+  __nv_bfloat16* Fz = reinterpret_cast<__nv_bfloat16*>(ws + w.Fz);
+  __nv_bfloat16* Yt = reinterpret_cast<__nv_bfloat16*>(ws + w.Yt);
+  float* part = reinterpret_cast<float*>(ws + w.tc_partial);
+  const double tol = 1e-6;
+
+  // tensor maps: X row tiles (rows_dot), X column tiles (cols_acc), and the three plane buffers
+  CUtensorMap tmA_rows, tmA_cols, tmD_rows, tmD_cols, tmFq, tmFz, tmYt;
+  const uint64_t sA = (uint64_t)L.strideA * 2, sD = (uint64_t)L.strideD * 2;
+  bool ok = make_tmap_bf16_3d(&tmA_rows, A, hi, N, S, (uint64_t)L.ldA * 2, sA, 64, 128) &&
+            make_tmap_bf16_3d(&tmA_cols, A, hi, N, S, (uint64_t)L.ldA * 2, sA, 64, 64) &&
+            make_tmap_bf16_3d(&tmD_rows, D, ho, N, S, (uint64_t)L.ldD * 2, sD, 64, 128) &&
+            make_tmap_bf16_3d(&tmD_cols, D, ho, N, S, (uint64_t)L.ldD * 2, sD, 64, 64) &&
+            make_tmap_bf16_3d(&tmFq, Fq, ho, rp, (uint64_t)S * 2, (uint64_t)ho * 2, (uint64_t)rp * ho * 2, 64, rp) &&
+            make_tmap_bf16_3d(&tmFz, Fz, hi, rp, (uint64_t)S * 2, (uint64_t)hi * 2, (uint64_t)rp * hi * 2, 64, rp) &&
+            make_tmap_bf16_3d(&tmYt, Yt, N, rp, (uint64_t)S * 2, (uint64_t)w.Npad * 2, (uint64_t)rp * w.Npad * 2, 64, rp);
+  if (!ok) return cudaErrorInvalidValue;
+
+  if (Q != Q0) DAD_STEP(cudaMemcpyAsync(Q, Q0, sizeof(float) * (size_t)S * r * ho, cudaMemcpyDeviceToDevice, st));
+  DAD_STEP(split_planes(Q0, S, r, ho, Fq, rp, st));
+  for (int k = 0; k < iters; ++k) {
+    DAD_STEP(umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st));                                  // Y = D G^T
+    DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, nullptr, nullptr, Fz, hi, part, ctr_cols, status, st));     // Z = Y^T A
+    DAD_STEP(umma_rows_dot(tmA_rows, tmFz, S, N, hi, r, Yt, w.Npad, status, st));                                  // W = A Z^T
+    DAD_STEP(umma_cols_acc(tmD_cols, tmYt, S, N, ho, r, Q, nullptr, nullptr, 0, part, ctr_cols, status, st));       // Gt = W^T D
+    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr,
+                                nullptr, 0, st));
+    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr, Fq,
+                                rp, st));
+  }
+  DAD_STEP(umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st));
+  DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, P, nullptr, nullptr, 0, part, ctr_cols, status, st));
+  if (sigma) DAD_STEP(row_norms<float>(P, (int64_t)S * r, hi, sigma, st));
+  return cudaSuccess;
+}
+
+static cudaError_t run_gemm_tc(const void* X, int64_t ldX, int64_t strideX, const void* Y, int64_t ldY, int64_t strideY,
+                               int S, int64_t N, int64_t hx, int64_t hy, float* C, char* ws, const GemmWs& w,
+                               cudaStream_t st) {
+  // the second status slot (byte 4) belongs to the dense products; the first keeps what a compress call reported
+  cudaError_t err = cudaMemsetAsync(ws + w.status + 4, 0, w.counters + w.n_counters * sizeof(unsigned) - w.status - 4, st);
+  if (err != cudaSuccess) return err;
+  CUtensorMap tmX, tmY;
+  if (!make_tmap_bf16_3d(&tmX, X, hx, N, S, (uint64_t)ldX * 2, (uint64_t)strideX * 2, 64, 64) ||
+      !make_tmap_bf16_3d(&tmY, Y, hy, N, S, (uint64_t)ldY * 2, (uint64_t)strideY * 2, 64, 64))
+    return cudaErrorInvalidValue;
+  return umma_gemm_tn(tmX, tmY, S, N, hx, hy, C, reinterpret_cast<float*>(ws + w.partial),
+                      reinterpret_cast<unsigned*>(ws + w.counters), reinterpret_cast<int*>(ws + w.status + 4), st);
+}
+
+#undef DAD_STEP
 
 }  // namespace dad
 
@@ -148,7 +267,10 @@ static dad_status validate_rank(const dad_layer* L, int r) {
 
 size_t dad_workspace_bytes(const dad_layer* L, int r, int iters) {
   if (validate_layer(L) != DAD_OK || validate_rank(L, r) != DAD_OK || iters < 0) return 0;
-  return compress_ws_layout(*L, r, L->dtype == DAD_F32).total;
+  const bool tc = tc_eligible(*L);
+  const size_t a = compress_ws_layout(*L, r, L->dtype == DAD_F32, tc).total;
+  const size_t b = tc ? gemm_ws_layout(L->h_in, L->h_out, L->S, L->N, false).total : 256;
+  return a > b ? a : b;
 }
 
 dad_status dad_full_grad(const dad_layer* L, const void* A, const void* D, float* grad, uint64_t* bytes_tx,
@@ -157,11 +279,17 @@ dad_status dad_full_grad(const dad_layer* L, const void* A, const void* D, float
   if (vs != DAD_OK) return vs;
   if (!A || !D || !grad) return DAD_ERR_NULL;
   if (!aligned(A, 16) || !aligned(D, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
-  (void)ws;
-  (void)ws_bytes;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  cudaError_t err = gemm_tn_simt(L->dtype, A, L->ldA, L->strideA, D, L->ldD, L->strideD, L->S, L->N, L->h_in,
-                                 L->h_out, grad, st);
+  cudaError_t err;
+  if (tc_eligible(*L)) {
+    const GemmWs w = gemm_ws_layout(L->h_in, L->h_out, L->S, L->N, false);
+    if (!ws) return DAD_ERR_NULL;
+    if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
+    if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
+    err = run_gemm_tc(A, L->ldA, L->strideA, D, L->ldD, L->strideD, L->S, L->N, L->h_in, L->h_out, grad, (char*)ws, w, st);
+  } else {
+    err = gemm_tn_simt(L->dtype, A, L->ldA, L->strideA, D, L->ldD, L->strideD, L->S, L->N, L->h_in, L->h_out, grad, st);
+  }
   if (err != cudaSuccess) return DAD_ERR_CUDA;
   if (bytes_tx)
     for (int s = 0; s < L->S; ++s) bytes_tx[s] = dad_bytes_dad(L);
@@ -180,11 +308,17 @@ dad_status dad_rank_compress(const dad_layer* L, const void* A, const void* D, i
       !aligned(ws, 256) || (sigma && !aligned(sigma, 4)))
     return DAD_ERR_ALIGN;
   const bool f64 = L->dtype == DAD_F32;
-  const CompressWs w = compress_ws_layout(*L, r, f64);
+  const bool tc = tc_eligible(*L);
+  const CompressWs w = compress_ws_layout(*L, r, f64, tc);
   if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  cudaError_t err = f64 ? run_compress<double>(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st)
-                        : run_compress<float>(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st);
+  cudaError_t err;
+  if (tc)
+    err = run_compress_tc(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st);
+  else if (f64)
+    err = run_compress<double>(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st);
+  else
+    err = run_compress<float>(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st);
   return err == cudaSuccess ? DAD_OK : DAD_ERR_CUDA;
 }
 
@@ -205,34 +339,48 @@ dad_status dad_gather_factors(const dad_layer* L, int r, const float* P, const f
   return DAD_OK;
 }
 
+static bool reconstruct_tc(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
+  return math == DAD_BF16 && h_in % 8 == 0 && h_out % 8 == 0 && K <= 0x7fffffff && tmap_encoder_available();
+}
+
 size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
-  (void)h_in;
-  (void)h_out;
-  (void)K;
-  (void)math;
-  return 0;
+  if (h_in < 1 || h_out < 1 || K < 1) return 0;
+  if (!reconstruct_tc(h_in, h_out, K, math)) return 0;
+  return gemm_ws_layout(h_in, h_out, 1, K, true).total;
 }
 
 dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat, float* grad,
                            dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream) {
-  if (h_in < 1 || h_out < 1 || K < 1) return DAD_ERR_SHAPE;
+  if (h_in < 1 || h_out < 1 || K < 1 || h_in > 0x7fffffff || h_out > 0x7fffffff) return DAD_ERR_SHAPE;
   if (math != DAD_F32 && math != DAD_BF16) return DAD_ERR_DTYPE;
   if (!Pcat || !Qcat || !grad) return DAD_ERR_NULL;
   if (!aligned(Pcat, 16) || !aligned(Qcat, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
-  if (ws_bytes < dad_reconstruct_workspace_bytes(h_in, h_out, K, math)) return DAD_ERR_WORKSPACE;
-  (void)ws;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  cudaError_t err = gemm_tn_simt(DAD_F32, Pcat, h_in, 0, Qcat, h_out, 0, 1, K, h_in, h_out, grad, st);
+  cudaError_t err;
+  if (reconstruct_tc(h_in, h_out, K, math)) {
+    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, K, true);
+    if (!ws) return DAD_ERR_NULL;
+    if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
+    if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
+    __nv_bfloat16* Xb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Xb);
+    __nv_bfloat16* Yb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Yb);
+    err = f32_to_bf16(Pcat, Xb, (size_t)K * h_in, st);
+    if (err == cudaSuccess) err = f32_to_bf16(Qcat, Yb, (size_t)K * h_out, st);
+    if (err == cudaSuccess) err = run_gemm_tc(Xb, h_in, K * h_in, Yb, h_out, K * h_out, 1, K, h_in, h_out, grad, (char*)ws, w, st);
+  } else {
+    err = gemm_tn_simt(DAD_F32, Pcat, h_in, 0, Qcat, h_out, 0, 1, K, h_in, h_out, grad, st);
+  }
   return err == cudaSuccess ? DAD_OK : DAD_ERR_CUDA;
 }
 
 dad_status dad_check(const void* ws, void* cuda_stream) {
   if (!ws) return DAD_ERR_NULL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  int status = 0;
-  if (cudaMemcpyAsync(&status, ws, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DAD_ERR_CUDA;
+  int status[2] = {0, 0};  // [0]: last dad_rank_compress on ws, [1]: last dense product on ws
+  if (cudaMemcpyAsync(status, ws, sizeof(status), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DAD_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return DAD_ERR_CUDA;
-  if (status == (int)DAD_ERR_TIMEOUT || status == (int)DAD_ERR_NUMERIC) return (dad_status)status;
+  for (int i = 0; i < 2; ++i)
+    if (status[i] == (int)DAD_ERR_TIMEOUT || status[i] == (int)DAD_ERR_NUMERIC) return (dad_status)status[i];
   return DAD_OK;
 }
 

@@ -2,6 +2,7 @@
 // layout of dad_rank_compress, and the host-side launchers of every kernel family.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
@@ -59,12 +60,26 @@ struct CompressWs {
   size_t gram;          // S*r*r doubles (Cholesky factor after the Gram kernel)
   size_t tratio;        // S*r doubles: R_jj / ||column|| after the first pass
   size_t dead;          // S*r bytes
-  // tensor-core pipeline: bf16 two-term splits of the small operands
-  size_t Fsplit;        // S*2*rp*max(h) bf16: split of the r x h factor operand (hi plane, lo plane)
-  size_t Ysplit;        // S*2*rp*Npad bf16: split of the N x r operand, stored transposed (rp x Npad)
+  // tensor-core pipeline: bf16 two-term (hi + lo) splits of the small fp32 operands
+  size_t Fq;            // S*2*rp*h_out bf16: planes of the iterate G (operand of D G^T)
+  size_t Fz;            // S*2*rp*h_in  bf16: planes of Z (operand of A Z^T)
+  size_t Yt;            // S*2*rp*Npad  bf16: planes of Y^T (operand of Y^T A and W^T D)
+  int64_t Npad;
+  size_t tc_partial;    // split partial tiles of the tensor-core column products
   size_t total;
 };
-CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64);
+// f64: fp64 pipeline (fp32 inputs); tc: tensor-core pipeline (bf16 inputs, 16-byte-aligned layout)
+CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc);
+
+// Workspace of dad_full_grad and of dad_reconstruct on the tensor cores.
+struct GemmWs {
+  size_t status, counters, n_counters, partial, Xb, Yb, total;  // Xb/Yb: bf16 copies of fp32 operands
+};
+GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands);
+
+// Whether the tensor-core kernels take this layer: bf16, all extents and strides multiples of 8
+// elements (TMA wants 16-byte strides), and the driver's tensor-map encoder is available.
+bool tc_eligible(const dad_layer& L);
 
 // ---- launchers (all asynchronous on `st`; return the first CUDA error) ------------------------
 // Y[s][n][j] = sum_c X[s][n][c] * F[s][j][c]      X: N x h (ld, site stride), F: r x h, Y: N x r
@@ -84,7 +99,7 @@ cudaError_t cols_acc(dad_dtype dt, const void* X, int64_t ld, int64_t stride, in
 template <typename T>
 cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, double* gram_partial,
                         double* gram, double* tratio, unsigned char* dead, unsigned* counters,
-                        int* status, float* out32, cudaStream_t st);
+                        int* status, float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
 
 // C[a][b] = sum_{s,n} X[s][n][a] * Y[s][n][b]  (fp32 FMA), C: hx x hy fp32 contiguous
 cudaError_t gemm_tn_simt(dad_dtype dt, const void* X, int64_t ldX, int64_t strideX, const void* Y,
@@ -96,5 +111,24 @@ cudaError_t copy_two(const float* a, float* a_out, size_t na, const float* b, fl
 cudaError_t widen_f32_to_f64(const float* in, double* out, size_t n, cudaStream_t st);
 template <typename T>
 cudaError_t row_norms(const T* M, int64_t rows, int64_t h, float* out, cudaStream_t st);
+// planes[s][0/1][j][c] = hi / lo bf16 terms of in[s][j][c]  (j < r; plane_rows >= r rows per plane)
+cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16* planes, int plane_rows,
+                         cudaStream_t st);
+cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStream_t st);
+
+// ---- tensor-core launchers (umma_gemm.cu) -------------------------------------------------------
+bool tmap_encoder_available();
+bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1_bytes,
+                       uint64_t s2_bytes, uint32_t box0, uint32_t box1);
+int umma_rank_pad(int r);
+int umma_cols_acc_splits(int S, int64_t N, int64_t h);
+int umma_gemm_splits(int64_t hx, int64_t hy, int64_t k_blocks);
+cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S, int64_t N, int64_t h, int r,
+                          __nv_bfloat16* yt_planes, int64_t ld_planes, int* status, cudaStream_t st);
+cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,
+                          float* out2, __nv_bfloat16* planes, int64_t ld_planes, float* partial, unsigned* counters,
+                          int* status, cudaStream_t st);
+cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, int S, int64_t N, int64_t hx, int64_t hy,
+                         float* C, float* partial, unsigned* counters, int* status, cudaStream_t st);
 
 }  // namespace dad

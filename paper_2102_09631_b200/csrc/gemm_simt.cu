@@ -119,6 +119,44 @@ cudaError_t widen_f32_to_f64(const float* in, double* out, size_t n, cudaStream_
   return err;
 }
 
+__global__ void split_planes_kernel(const float* __restrict__ in, int r, int64_t h, __nv_bfloat16* __restrict__ planes,
+                                    int plane_rows, size_t n) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const size_t c = i % (size_t)h, sj = i / (size_t)h;
+    const size_t j = sj % (size_t)r, s = sj / (size_t)r;
+    const float f = in[i];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(f);
+    planes[((s * 2 + 0) * plane_rows + j) * h + c] = hi;
+    planes[((s * 2 + 1) * plane_rows + j) * h + c] = __float2bfloat16_rn(f - __bfloat162float(hi));
+  }
+}
+
+cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16* planes, int plane_rows,
+                         cudaStream_t st) {
+  cudaError_t err = cudaSuccess;
+  const size_t n = (size_t)S * r * h;
+  size_t blocks = (n + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  DAD_LAUNCH(err, "split_planes", split_planes_kernel, (unsigned)blocks, 256, 0, st, in, r, h, planes, plane_rows, n);
+  return err;
+}
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, size_t n) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
+}
+
+cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStream_t st) {
+  cudaError_t err = cudaSuccess;
+  size_t blocks = (n + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  DAD_LAUNCH(err, "f32_to_bf16", f32_to_bf16_kernel, (unsigned)blocks, 256, 0, st, in, out, n);
+  return err;
+}
+
 // out[row] = || M[row] ||_2, one warp per row (sigma_j = ||P_j||, Algorithm 2's sqrt(v^T C v)).
 template <typename T>
 __global__ void __launch_bounds__(256) row_norms_kernel(const T* __restrict__ M, int64_t rows, int64_t h,

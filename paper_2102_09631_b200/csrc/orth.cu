@@ -120,7 +120,8 @@ gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int 
 template <typename T>
 __global__ void __launch_bounds__(128)
 tri_solve_kernel(T* __restrict__ G, int r, int64_t h, const double* __restrict__ L,
-                 const unsigned char* __restrict__ dead, float* __restrict__ out32) {
+                 const unsigned char* __restrict__ dead, float* __restrict__ out32,
+                 __nv_bfloat16* __restrict__ planes, int plane_rows) {
   extern __shared__ double sm[];  // r*r (L) + r*128 (solved column values)
   double* Ls = sm;
   double* qs = sm + r * r;
@@ -138,13 +139,19 @@ tri_solve_kernel(T* __restrict__ G, int r, int64_t h, const double* __restrict__
     qs[j * 128 + tid] = v;
     Gs[(int64_t)j * h + b] = (T)v;
     if (out32) out32[((int64_t)s * r + j) * h + b] = (float)v;
+    if (planes) {  // hi + lo bf16 terms of the fp32 value, for the tensor-core product that reads it next
+      const float f = (float)v;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(f);
+      planes[(((int64_t)s * 2 + 0) * plane_rows + j) * h + b] = hi;
+      planes[(((int64_t)s * 2 + 1) * plane_rows + j) * h + b] = __float2bfloat16_rn(f - __bfloat162float(hi));
+    }
   }
 }
 
 template <typename T>
 cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, double* gram_partial,
                         double* gram, double* tratio, unsigned char* dead, unsigned* counters,
-                        int* status, float* out32, cudaStream_t st) {
+                        int* status, float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st) {
   cudaError_t err = cudaSuccess;
   const int chunks = (int)ceil_div(h, kGramChunk);
   const int a = r * (kGramChunk + 1), b = r * (r + 1);
@@ -158,12 +165,12 @@ cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, dou
   DAD_LAUNCH(err, "gram_cholesky", (gram_cholesky_kernel<T>), dim3((unsigned)chunks, (unsigned)S), 256, smem1, st, G, r, h, chunks, pass,
              tol, gram_partial, gram, tratio, dead, counters, status);
   DAD_LAUNCH(err, "tri_solve", (tri_solve_kernel<T>), dim3((unsigned)ceil_div(h, 128), (unsigned)S), 128, smem2, st, G, r, h, gram,
-             dead, out32);
+             dead, out32, planes, plane_rows);
   return err;
 }
 template cudaError_t cholqr_pass<float>(float*, int, int, int64_t, int, double, double*, double*, double*,
-                                        unsigned char*, unsigned*, int*, float*, cudaStream_t);
+                                        unsigned char*, unsigned*, int*, float*, __nv_bfloat16*, int, cudaStream_t);
 template cudaError_t cholqr_pass<double>(double*, int, int, int64_t, int, double, double*, double*, double*,
-                                         unsigned char*, unsigned*, int*, float*, cudaStream_t);
+                                         unsigned char*, unsigned*, int*, float*, __nv_bfloat16*, int, cudaStream_t);
 
 }  // namespace dad

@@ -1,0 +1,415 @@
+// Tensor-core (tcgen05 / TMEM) kernel family for bf16 inputs.  One kernel template computes a
+// 128 x BN tile  D[m][n] = sum_k Aop[m][k] * Bop[n][k]  with fp32 accumulation in tensor memory,
+// operands staged by TMA into 128-byte-swizzled shared memory behind an mbarrier ring:
+//
+//   rows_dot  Y = X F^T     (Eq. "reduced_iter", the products D g and A z of a power iteration):
+//             A operand = X tile, K-major (row-major X, contraction along its columns);
+//             B operand = the r x h factor as two bf16 planes (hi + lo split of fp32), K-major.
+//             Epilogue writes Y transposed as bf16 hi/lo planes, the layout cols_acc reads.
+//   cols_acc  Z = Y^T X     (the products A^T v and D^T w):
+//             A operand = X tile read as its transpose, M/N-major (contraction along rows);
+//             B operand = Y^T planes, K-major.  Rows are split over CTAs; partial tiles are summed
+//             in split order by the last CTA to arrive (deterministic).  Epilogue writes Z as fp32
+//             and, if asked, as bf16 hi/lo planes for the next rows_dot.
+//   gemm_tn   C = X^T Y     (the dAD gradient sum_s A_s^T D_s of Sec. 3.2 and the reconstruction
+//             Pcat^T Qcat of Algorithm 1): both operands M/N-major, optional split over the
+//             contraction with the same ordered reduction.
+//
+// Warp roles (192 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
+// MMAs, warps 2-5 drain the accumulator (each warp reads its own quarter of the 128 TMEM lanes).
+// Every mbarrier wait is bounded; if one runs out the CTA raises an abort flag, all roles leave
+// their loops, outstanding copies are waited for (bounded), tensor memory is freed, and the status
+// word in the workspace is set to DAD_ERR_TIMEOUT.
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace dad {
+using namespace sm100;
+
+enum : int { EPI_YT = 0, EPI_Z = 1, EPI_C = 2 };
+
+struct UmmaParams {
+  int m_extent;      // valid rows of D: N (rows_dot), h (cols_acc), h_in (gemm_tn)
+  int n_extent;      // valid columns of D: r, or h_out
+  int k_blocks;      // 64-wide blocks of the contraction (per batch entry)
+  int kb_per_split;
+  int splits;
+  int kb_per_site;   // gemm_tn over sites: blocks per site (site = block / kb_per_site); 0 = batch from blockIdx.z
+  float* out_f32;    // EPI_Z: [batch][r][ld_out];  EPI_C: [m][ld_out]
+  float* out2_f32;   // EPI_Z: optional second copy, same layout
+  int64_t ld_out;
+  __nv_bfloat16* out_planes;  // EPI_YT / EPI_Z: [batch][2][plane_rows][ld_planes] (hi plane, lo plane), or null
+  int64_t ld_planes;
+  int plane_rows;    // rows per plane (r rounded up to the MMA width); rows >= r are never written
+  float* partial;    // split partial tiles [tile][split][128][BN]
+  unsigned* counters;
+  int* status;
+};
+
+template <int BN, bool A_MN, bool B_MN, int TERMS, int EPI, int STAGES>
+__global__ void __launch_bounds__(192)
+umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const UmmaParams p) {
+  constexpr int A_BYTES = 128 * 64 * 2;
+  constexpr int B_BYTES = B_MN ? (BN / 64) * 8192 : TERMS * BN * 128;
+  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+  constexpr uint32_t IDESC = instr_desc(128, BN, A_MN, B_MN);
+  static_assert(!B_MN || (BN % 64 == 0 && TERMS == 1), "M/N-major B comes in 64-wide chunks, one term");
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag, issued_s, last_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tile = blockIdx.x;
+  const int n_tile = blockIdx.y / p.splits, split = blockIdx.y % p.splits;
+  const int batch = blockIdx.z;
+  const int m0 = m_tile * 128, n0 = n_tile * BN;
+  const int kb0 = split * p.kb_per_split;
+  const int kb1 = (kb0 + p.kb_per_split < p.k_blocks) ? kb0 + p.kb_per_split : p.k_blocks;
+  const int nkb = kb1 > kb0 ? kb1 - kb0 : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&accum_bar, 1);
+    abort_flag = 0;
+    issued_s = 0;
+    last_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_s, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmA);
+      prefetch_tmap(&tmB);
+      int i = 0;
+      for (; i < nkb; ++i) {
+        const int stage = i % STAGES;
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp)) break;
+        mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+        uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
+        uint8_t* b_dst = a_dst + A_BYTES;
+        const int kb = kb0 + i;
+        int kcoord = kb * 64, bz = batch;
+        if (p.kb_per_site > 0) {
+          bz = kb / p.kb_per_site;
+          kcoord = (kb % p.kb_per_site) * 64;
+        }
+        if constexpr (A_MN) {
+          tma_load_3d(a_dst, &tmA, &full_bar[stage], m0, kcoord, bz);
+          tma_load_3d(a_dst + 8192, &tmA, &full_bar[stage], m0 + 64, kcoord, bz);
+        } else {
+          tma_load_3d(a_dst, &tmA, &full_bar[stage], kcoord, m0, bz);
+        }
+        if constexpr (B_MN) {
+#pragma unroll
+          for (int c = 0; c < BN / 64; ++c) tma_load_3d(b_dst + c * 8192, &tmB, &full_bar[stage], n0 + c * 64, kcoord, bz);
+        } else {
+#pragma unroll
+          for (int t = 0; t < TERMS; ++t) tma_load_3d(b_dst + t * BN * 128, &tmB, &full_bar[stage], kcoord, n0, bz * TERMS + t);
+        }
+        issued_s = i + 1;
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      for (int i = 0; i < nkb; ++i) {
+        const int stage = i % STAGES;
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        if (!mbar_wait(&full_bar[stage], ph, abortp)) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+        const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+        for (int k16 = 0; k16 < 4; ++k16) {
+          const uint64_t adesc = A_MN ? desc_mn_major(a_addr, k16) : desc_k_major(a_addr, k16);
+#pragma unroll
+          for (int t = 0; t < TERMS; ++t) {
+            const uint64_t bdesc = B_MN ? desc_mn_major(b_addr, k16) : desc_k_major(b_addr + t * BN * 128, k16);
+            umma_bf16(tmem_base, adesc, bdesc, IDESC, (i | k16 | t) != 0 ? 1u : 0u);
+          }
+        }
+        umma_commit(&empty_bar[stage]);
+      }
+      umma_commit(&accum_bar);
+    }
+  } else {
+    // ---- epilogue: 4 warps, warp (id % 4) owns TMEM lanes 32*(id % 4) .. +31 ----
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+    const bool ok = mbar_wait(&accum_bar, 0u, abortp);
+    tc_fence_after();
+    const int tiles_n = gridDim.y / p.splits;
+    const int64_t tile_lin = ((int64_t)batch * gridDim.x + m_tile) * tiles_n + n_tile;
+    float* my_partial = p.partial ? p.partial + ((tile_lin * p.splits + split) * 128 + row) * BN : nullptr;
+    bool finish = ok;
+    if (ok && p.splits > 1) {
+#pragma unroll 1
+      for (int c = 0; c < BN / 16; ++c) {
+        float v[16];
+        if (nkb > 0) {
+          tmem_ld16(lane_base + c * 16, v);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
+        float4* dst = reinterpret_cast<float4*>(my_partial + c * 16);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+      }
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (warp == 2 && lane == 0) {
+        unsigned* ctr = p.counters + tile_lin;
+        const unsigned old = atomicAdd(ctr, 1u);
+        const int is_last = (old == (unsigned)p.splits - 1u);
+        if (is_last) *ctr = 0u;
+        last_flag = is_last;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      finish = last_flag != 0;
+      if (finish) __threadfence();
+    }
+    if (finish) {
+      const int64_t gm = (int64_t)m0 + row;  // global row of D
+#pragma unroll 1
+      for (int c = 0; c < BN / 16; ++c) {
+        float v[16];
+        if (p.splits > 1) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0.f;
+          const float* src = p.partial + (tile_lin * p.splits * 128 + row) * BN + c * 16;
+          for (int s = 0; s < p.splits; ++s) {
+            const float4* s4 = reinterpret_cast<const float4*>(src + (int64_t)s * 128 * BN);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 t = __ldcg(s4 + i);
+              v[4 * i] += t.x;
+              v[4 * i + 1] += t.y;
+              v[4 * i + 2] += t.z;
+              v[4 * i + 3] += t.w;
+            }
+          }
+        } else if (nkb > 0) {
+          tmem_ld16(lane_base + c * 16, v);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
+        if (gm < p.m_extent) {
+          if constexpr (EPI == EPI_C) {
+            float* dst = p.out_f32 + gm * p.ld_out + n0 + c * 16;
+            if (n0 + c * 16 + 16 <= p.n_extent && (p.ld_out & 3) == 0) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                if (n0 + c * 16 + i < p.n_extent) dst[i] = v[i];
+            }
+          } else {
+            const int r = p.n_extent;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int j = c * 16 + i;
+              if (j < r) {
+                if constexpr (EPI == EPI_Z) {
+                  if (p.out_f32) p.out_f32[((int64_t)batch * r + j) * p.ld_out + gm] = v[i];
+                  if (p.out2_f32) p.out2_f32[((int64_t)batch * r + j) * p.ld_out + gm] = v[i];
+                }
+                if (p.out_planes) {
+                  const __nv_bfloat16 hi = __float2bfloat16_rn(v[i]);
+                  const __nv_bfloat16 lo = __float2bfloat16_rn(v[i] - __bfloat162float(hi));
+                  p.out_planes[(((int64_t)batch * 2 + 0) * p.plane_rows + j) * p.ld_planes + gm] = hi;
+                  p.out_planes[(((int64_t)batch * 2 + 1) * p.plane_rows + j) * p.ld_planes + gm] = lo;
+                }
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    if (threadIdx.x == 0) {
+      // wait (bounded) for copies already issued into this CTA's shared memory
+      const int issued = issued_s;
+      const int first = issued > STAGES ? issued - STAGES : 0;
+      for (int i = first; i < issued; ++i) {
+        uint64_t* bar = &full_bar[i % STAGES];
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(bar, ph); ++t) {
+        }
+      }
+      if (p.status) *p.status = (int)DAD_ERR_TIMEOUT;
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+bool tmap_encoder_available() { return encode_fn() != nullptr; }
+
+// bf16 tensor (d0 innermost, contiguous) x d1 x d2 with byte strides s1, s2; box = box0 x box1 x 1,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1_bytes,
+                       uint64_t s2_bytes, uint32_t box0, uint32_t box1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  if (d2 <= 1 && s2_bytes < s1_bytes) s2_bytes = s1_bytes * d1;
+  cuuint64_t strides[2] = {s1_bytes, s2_bytes};
+  cuuint32_t box[3] = {box0, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int umma_rank_pad(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
+
+int umma_cols_acc_splits(int S, int64_t N, int64_t h) {
+  const int64_t tiles = ceil_div(h, 128) * S;
+  const int64_t kb = ceil_div(N, 64);
+  int64_t splits = ceil_div(148 * 3, tiles);
+  if (splits > kb / 4) splits = kb / 4;  // at least 4 blocks (256 rows) per split
+  if (splits > 16) splits = 16;
+  if (splits < 1) splits = 1;
+  const int64_t per = ceil_div(kb, splits);
+  return (int)ceil_div(kb, per);  // no empty split
+}
+
+template <int BN, bool A_MN, bool B_MN, int TERMS, int EPI, int STAGES>
+static cudaError_t launch_umma(const CUtensorMap& tmA, const CUtensorMap& tmB, const UmmaParams& p, dim3 grid,
+                               const char* tag, cudaStream_t st) {
+  constexpr int A_BYTES = 128 * 64 * 2;
+  constexpr int B_BYTES = B_MN ? (BN / 64) * 8192 : TERMS * BN * 128;
+  constexpr size_t smem = (size_t)STAGES * (A_BYTES + B_BYTES) + 1024;
+  auto kernel = umma_kernel<BN, A_MN, B_MN, TERMS, EPI, STAGES>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  DAD_LAUNCH(err, tag, kernel, grid, 192, smem, st, tmA, tmB, p);
+  return err;
+}
+
+// Y^T planes <- split(X F^T).  tmX: X as (h, N, S) with box 64 x 128; tmF: factor planes as (h, rp, 2S) with box 64 x rp,
+// rp = umma_rank_pad(r).
+cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S, int64_t N, int64_t h, int r,
+                          __nv_bfloat16* yt_planes, int64_t ld_planes, int* status, cudaStream_t st) {
+  UmmaParams p{};
+  p.m_extent = (int)N;
+  p.n_extent = r;
+  p.k_blocks = (int)ceil_div(h, 64);
+  p.kb_per_split = p.k_blocks;
+  p.splits = 1;
+  p.out_planes = yt_planes;
+  p.ld_planes = ld_planes;
+  p.plane_rows = umma_rank_pad(r);
+  p.status = status;
+  dim3 grid((unsigned)ceil_div(N, 128), 1, (unsigned)S);
+  switch (umma_rank_pad(r)) {
+    case 16: return launch_umma<16, false, false, 2, EPI_YT, 5>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    case 32: return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    default: return launch_umma<64, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
+  }
+}
+
+// Z <- Y^T X.  tmX: X as (h, N, S) with box 64 x 64; tmYt: Y^T planes as (N, rp, 2S) with box 64 x rp.
+cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,
+                          float* out2, __nv_bfloat16* planes, int64_t ld_planes, float* partial, unsigned* counters,
+                          int* status, cudaStream_t st) {
+  UmmaParams p{};
+  p.m_extent = (int)h;
+  p.n_extent = r;
+  p.k_blocks = (int)ceil_div(N, 64);
+  p.splits = umma_cols_acc_splits(S, N, h);
+  p.kb_per_split = (int)ceil_div(p.k_blocks, p.splits);
+  p.out_f32 = out;
+  p.out2_f32 = out2;
+  p.ld_out = h;
+  p.out_planes = planes;
+  p.ld_planes = ld_planes;
+  p.plane_rows = umma_rank_pad(r);
+  p.partial = partial;
+  p.counters = counters;
+  p.status = status;
+  dim3 grid((unsigned)ceil_div(h, 128), (unsigned)p.splits, (unsigned)S);
+  switch (umma_rank_pad(r)) {
+    case 16: return launch_umma<16, true, false, 2, EPI_Z, 5>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+    case 32: return launch_umma<32, true, false, 2, EPI_Z, 4>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+    default: return launch_umma<64, true, false, 2, EPI_Z, 4>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+  }
+}
+
+int umma_gemm_splits(int64_t hx, int64_t hy, int64_t k_blocks) {
+  const int64_t tiles = ceil_div(hx, 128) * ceil_div(hy, 128);
+  int64_t splits = 148 / tiles;
+  if (splits > k_blocks / 8) splits = k_blocks / 8;
+  if (splits > 32) splits = 32;
+  if (splits < 1) splits = 1;
+  const int64_t per = ceil_div(k_blocks, splits);
+  return (int)ceil_div(k_blocks, per);
+}
+
+// C (hx x hy, fp32) <- sum over sites and rows of X^T Y.  tmX: (hx, N, S) box 64 x 64; tmY: (hy, N, S) box 64 x 64.
+cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, int S, int64_t N, int64_t hx, int64_t hy,
+                         float* C, float* partial, unsigned* counters, int* status, cudaStream_t st) {
+  UmmaParams p{};
+  p.m_extent = (int)hx;
+  p.n_extent = (int)hy;
+  p.kb_per_site = (int)ceil_div(N, 64);
+  p.k_blocks = p.kb_per_site * S;
+  p.splits = umma_gemm_splits(hx, hy, p.k_blocks);
+  p.kb_per_split = (int)ceil_div(p.k_blocks, p.splits);
+  p.out_f32 = C;
+  p.ld_out = hy;
+  p.partial = partial;
+  p.counters = counters;
+  p.status = status;
+  dim3 grid((unsigned)ceil_div(hx, 128), (unsigned)(ceil_div(hy, 128) * p.splits), 1);
+  return launch_umma<128, true, true, 1, EPI_C, 6>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+}
+
+}  // namespace dad
