@@ -38,6 +38,8 @@ def parse_args():
     ap.add_argument("--iters", type=int, default=None, help="override the power-iteration count")
     ap.add_argument("--resident-blocks", type=int, default=4,
                     help="distinct transformer blocks of input data kept in HBM and cycled through")
+    ap.add_argument("--blocks", type=int, default=None,
+                    help="run only this many of the network's blocks per step (profiling captures); default all")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -203,6 +205,9 @@ def run_ours(args):
     B.lib()
 
     cfg = wl.CONFIGS[args.config]
+    if args.blocks is not None:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, blocks=max(1, min(cfg.blocks, args.blocks)))
     r = args.rank or cfg.r
     iters = cfg.iters if args.iters is None else args.iters
     layers = expand_layers(cfg)

@@ -71,7 +71,7 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc) {
   w.tratio = off;
   off = align_up(off + S * rr * 8, 256);
   w.dead = off;
-  off = align_up(off + S * rr, 256);
+  off = align_up(off + align_up(S * rr, 16) + S * sizeof(int), 256);
   w.Fq = w.Fz = w.Yt = w.tc_partial = off;
   if (tc) {
     const size_t rp = (size_t)umma_rank_pad(r);
@@ -141,6 +141,7 @@ static cudaError_t run_compress(const dad_layer& L, const void* A, const void* D
   double* gram = reinterpret_cast<double*>(ws + w.gram);
   double* tratio = reinterpret_cast<double*>(ws + w.tratio);
   unsigned char* dead = reinterpret_cast<unsigned char*>(ws + w.dead);
+  int* need2 = reinterpret_cast<int*>(ws + w.dead + align_up((size_t)S * r, 16));
   const double tol = f64 ? 1e-12 : 1e-6;
   TAcc* G;
   if constexpr (f64) {
@@ -158,11 +159,12 @@ static cudaError_t run_compress(const dad_layer& L, const void* A, const void* D
     DAD_STEP(cols_acc<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Y, r, Z, nullptr, part, ctr_cols, st));  // Z = Y^T A
     DAD_STEP(rows_dot<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Z, r, Y, st));                           // W = A Z^T
     DAD_STEP(cols_acc<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, Y, r, G, nullptr, part, ctr_cols, st));  // Gt = W^T D
-    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr,
-                               nullptr, 0, st));
+    // the second pass returns at once for sites whose first pass was well conditioned, so both write the outputs
     float* q32 = (f64 && k == iters - 1) ? Q : nullptr;
-    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, ctr_gram, status, q32, nullptr,
-                               0, st));
+    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,
+                               nullptr, 0, st));
+    DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,
+                               nullptr, 0, st));
   }
   DAD_STEP(rows_dot<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, G, r, Y, st));
   DAD_STEP(cols_acc<TAcc>(L.dtype, A, L.ldA, L.strideA, S, N, hi, Y, r, Z, P, part, ctr_cols, st));
@@ -186,6 +188,7 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
   double* gram = reinterpret_cast<double*>(ws + w.gram);
   double* tratio = reinterpret_cast<double*>(ws + w.tratio);
   unsigned char* dead = reinterpret_cast<unsigned char*>(ws + w.dead);
+  int* need2 = reinterpret_cast<int*>(ws + w.dead + align_up((size_t)S * r, 16));
   __nv_bfloat16* Fq = reinterpret_cast<__nv_bfloat16*>(ws + w.Fq);
   __nv_bfloat16* Fz = reinterpret_cast<__nv_bfloat16*>(ws + w.Fz);
   __nv_bfloat16* Yt = reinterpret_cast<__nv_bfloat16*>(ws + w.Yt);
@@ -211,10 +214,10 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
     DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, nullptr, nullptr, Fz, hi, part, ctr_cols, status, st));     // Z = Y^T A
     DAD_STEP(umma_rows_dot(tmA_rows, tmFz, S, N, hi, r, Yt, w.Npad, status, st));                                  // W = A Z^T
     DAD_STEP(umma_cols_acc(tmD_cols, tmYt, S, N, ho, r, Q, nullptr, nullptr, 0, part, ctr_cols, status, st));       // Gt = W^T D
-    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr,
-                                nullptr, 0, st));
-    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, ctr_gram, status, nullptr, Fq,
-                                rp, st));
+    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, nullptr,
+                                Fq, rp, st));
+    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, nullptr,
+                                Fq, rp, st));
   }
   DAD_STEP(umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st));
   DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, P, nullptr, nullptr, 0, part, ctr_cols, status, st));

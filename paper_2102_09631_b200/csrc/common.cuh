@@ -59,7 +59,7 @@ struct CompressWs {
   size_t gram_partial;  // S*chunks*r*r doubles
   size_t gram;          // S*r*r doubles (Cholesky factor after the Gram kernel)
   size_t tratio;        // S*r doubles: R_jj / ||column|| after the first pass
-  size_t dead;          // S*r bytes
+  size_t dead;          // S*r bytes, then S ints: whether the site needs the second pass
   // tensor-core pipeline: bf16 two-term (hi + lo) splits of the small fp32 operands
   size_t Fq;            // S*2*rp*h_out bf16: planes of the iterate G (operand of D G^T)
   size_t Fz;            // S*2*rp*h_in  bf16: planes of Z (operand of A Z^T)
@@ -98,7 +98,7 @@ cudaError_t cols_acc(dad_dtype dt, const void* X, int64_t ld, int64_t stride, in
 // remainder is <= tol of their length.  out32 (optional) receives an fp32 copy of the result.
 template <typename T>
 cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, double* gram_partial,
-                        double* gram, double* tratio, unsigned char* dead, unsigned* counters,
+                        double* gram, double* tratio, unsigned char* dead, int* need2, unsigned* counters,
                         int* status, float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
 
 // C[a][b] = sum_{s,n} X[s][n][a] * Y[s][n][b]  (fp32 FMA), C: hx x hy fp32 contiguous

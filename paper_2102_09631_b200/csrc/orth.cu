@@ -2,30 +2,36 @@
 // Eq. "peel": each vector loses its components along the ones before it), as Cholesky-QR:
 //   Gram = G G^T (fp64, r x r)  ->  Gram = L L^T  ->  rows of G <- L^{-1} G.
 // This is the thin QR with positive diagonal (R = L^T).  One pass leaves an orthogonality
-// defect of about 1e-16 * cond(G)^2, so the pass is applied twice.  Pivots are kept from
-// collapsing: a pivot below (1e-7)^2 of the vector's squared length is raised to that value in
-// the first pass (the vector then comes out short instead of wrong), and the second pass, which
-// sees a well-conditioned matrix, decides from the product of both passes' diagonals whether the
-// vector carried any new direction; if not it is set to exactly zero.
+// defect of about 1e-16 * cond(G)^2, so a second pass follows whenever the first one shows that
+// some vector lost more than three digits to the projection (R_jj < 1e-3 ||g_j||); otherwise the
+// second pass's kernels return at once.  Pivots are kept from collapsing: a pivot below (1e-7)^2
+// of the vector's squared length is raised to that value in the first pass (the vector then comes
+// out short instead of wrong), and the second pass, which sees a well-conditioned matrix, decides
+// from the product of both passes' diagonals whether the vector carried any new direction; if not
+// it is set to exactly zero.
 #include "common.cuh"
 
 namespace dad {
 
-constexpr double kPivotFloor = 1e-14;  // (1e-7)^2, relative to the squared length of the vector
+constexpr double kPivotFloor = 1e-14;   // (1e-7)^2, relative to the squared length of the vector
+constexpr double kSecondPassBelow = 1e-3;
 
 template <typename T>
 __global__ void __launch_bounds__(256)
 gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int pass, double tol,
                      double* __restrict__ partial, double* __restrict__ Lout, double* __restrict__ tratio,
-                     unsigned char* __restrict__ dead, unsigned* __restrict__ counters, int* __restrict__ status) {
-  extern __shared__ double sm[];  // max(r * (kGramChunk + 1), r * (r + 1)) doubles
+                     unsigned char* __restrict__ dead, int* __restrict__ need2, unsigned* __restrict__ counters,
+                     int* __restrict__ status) {
+  extern __shared__ double sm[];  // tile of T [r][kGramChunk + 1], later the r x (r + 1) factor in fp64
   const int s = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
+  if (pass == 1 && need2[s] == 0) return;
+  T* tile = reinterpret_cast<T*>(sm);
   const T* Gs = G + (int64_t)s * r * h;
   const int64_t c0 = (int64_t)chunk * kGramChunk;
   constexpr int LD = kGramChunk + 1;
   for (int idx = tid; idx < r * kGramChunk; idx += 256) {
     const int j = idx / kGramChunk, cc = idx % kGramChunk;
-    sm[j * LD + cc] = (c0 + cc < h) ? (double)Gs[(int64_t)j * h + c0 + cc] : 0.0;
+    tile[j * LD + cc] = (c0 + cc < h) ? Gs[(int64_t)j * h + c0 + cc] : T(0);
   }
   __syncthreads();
   double* mine = partial + ((int64_t)s * chunks + chunk) * r * r;
@@ -34,7 +40,7 @@ gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int 
     if (j <= i) {
       double acc = 0.0;
 #pragma unroll 8
-      for (int cc = 0; cc < kGramChunk; ++cc) acc += sm[i * LD + cc] * sm[j * LD + cc];
+      for (int cc = 0; cc < kGramChunk; ++cc) acc += (double)tile[i * LD + cc] * (double)tile[j * LD + cc];
       mine[p] = acc;
     }
   }
@@ -49,26 +55,36 @@ gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int 
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  // Sum the chunk partials in chunk order, then factor in shared memory.
+  // Sum the chunk partials in chunk order (loads issued eight at a time), then factor in shared memory.
   const int LR = r + 1;
   const double* src = partial + (int64_t)s * chunks * r * r;
+  const int64_t rr = (int64_t)r * r;
   for (int p = tid; p < r * r; p += 256) {
     const int i = p / r, j = p % r;
     if (j <= i) {
       double v = 0.0;
-      for (int q = 0; q < chunks; ++q) v += __ldcg(src + (int64_t)q * r * r + p);
+      int q = 0;
+      for (; q + 8 <= chunks; q += 8) {
+        double t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) t[u] = __ldcg(src + (q + u) * rr + p);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v += t[u];
+      }
+      for (; q < chunks; ++q) v += __ldcg(src + q * rr + p);
       sm[i * LR + j] = v;
     }
   }
   __shared__ double ljj;
   __shared__ int col_dead;
+  __shared__ double min_ratio;
+  if (tid == 0) min_ratio = 1.0;
   __syncthreads();
   double* Ls = Lout + (int64_t)s * r * r;
   for (int j = 0; j < r; ++j) {
     if (tid == 0) {
-      // the squared length of vector j before projection is its Gram diagonal: kept in tratio/dead bookkeeping
       const double d = sm[j * LR + j];
-      // original diagonal = d + sum_l L_jl^2
+      // squared length of vector j before projection = remaining pivot + what the earlier columns took
       double orig = d;
       for (int l = 0; l < j; ++l) orig += sm[j * LR + l] * sm[j * LR + l];
       int is_dead = 0;
@@ -82,10 +98,12 @@ gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int 
         const double floor_ = kPivotFloor * orig;
         if (!(piv > floor_)) piv = floor_;
       }
-      double l = is_dead ? 1.0 : sqrt(piv);
+      const double l = is_dead ? 1.0 : sqrt(piv);
       if (!is_dead) {
         if (pass == 0) {
-          tratio[(int64_t)s * r + j] = l / sqrt(orig);
+          const double t = l / sqrt(orig);
+          tratio[(int64_t)s * r + j] = t;
+          if (t < min_ratio) min_ratio = t;
         } else {
           // total remainder relative to the vector's length before the first pass
           const double total = tratio[(int64_t)s * r + j] * l;
@@ -115,25 +133,29 @@ gram_cholesky_kernel(const T* __restrict__ G, int r, int64_t h, int chunks, int 
     const int i = p / r, j = p % r;
     Ls[p] = (j <= i) ? sm[i * LR + j] : 0.0;
   }
+  if (tid == 0 && pass == 0) need2[s] = (min_ratio < kSecondPassBelow) ? 1 : 0;
 }
 
 template <typename T>
 __global__ void __launch_bounds__(128)
-tri_solve_kernel(T* __restrict__ G, int r, int64_t h, const double* __restrict__ L,
-                 const unsigned char* __restrict__ dead, float* __restrict__ out32,
+tri_solve_kernel(T* __restrict__ G, int r, int64_t h, int pass, const double* __restrict__ L,
+                 const unsigned char* __restrict__ dead, const int* __restrict__ need2, float* __restrict__ out32,
                  __nv_bfloat16* __restrict__ planes, int plane_rows) {
-  extern __shared__ double sm[];  // r*r (L) + r*128 (solved column values)
+  extern __shared__ double sm[];  // r*r (L) + r*128 (column values, solved in place)
   double* Ls = sm;
   double* qs = sm + r * r;
   const int s = blockIdx.y, tid = threadIdx.x;
+  if (pass == 1 && need2[s] == 0) return;
+  const int64_t b = (int64_t)blockIdx.x * 128 + tid;
+  T* Gs = G + (int64_t)s * r * h;
+  if (b < h)
+    for (int j = 0; j < r; ++j) qs[j * 128 + tid] = (double)Gs[(int64_t)j * h + b];  // independent loads, all in flight
   for (int p = tid; p < r * r; p += 128) Ls[p] = L[(int64_t)s * r * r + p];
   __syncthreads();
-  const int64_t b = (int64_t)blockIdx.x * 128 + tid;
   if (b >= h) return;
-  T* Gs = G + (int64_t)s * r * h;
   const unsigned char* ds = dead + (int64_t)s * r;
   for (int j = 0; j < r; ++j) {
-    double v = (double)Gs[(int64_t)j * h + b];
+    double v = qs[j * 128 + tid];
     for (int l = 0; l < j; ++l) v -= Ls[j * r + l] * qs[l * 128 + tid];
     v = ds[j] ? 0.0 : v / Ls[j * r + j];
     qs[j * 128 + tid] = v;
@@ -150,27 +172,33 @@ tri_solve_kernel(T* __restrict__ G, int r, int64_t h, const double* __restrict__
 
 template <typename T>
 cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, double* gram_partial,
-                        double* gram, double* tratio, unsigned char* dead, unsigned* counters,
+                        double* gram, double* tratio, unsigned char* dead, int* need2, unsigned* counters,
                         int* status, float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st) {
   cudaError_t err = cudaSuccess;
   const int chunks = (int)ceil_div(h, kGramChunk);
-  const int a = r * (kGramChunk + 1), b = r * (r + 1);
-  const size_t smem1 = sizeof(double) * (size_t)(a > b ? a : b);
+  const size_t a = sizeof(T) * (size_t)r * (kGramChunk + 1), b = sizeof(double) * (size_t)r * (r + 1);
+  const size_t smem1 = a > b ? a : b;
   const size_t smem2 = sizeof(double) * (size_t)(r * r + r * 128);
   // the opt-in is per device and cheap, so it is simply made on every call
+  if (smem1 > 48 * 1024) {
+    err = cudaFuncSetAttribute(gram_cholesky_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    if (err != cudaSuccess) return err;
+  }
   if (smem2 > 48 * 1024) {
     err = cudaFuncSetAttribute(tri_solve_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
     if (err != cudaSuccess) return err;
   }
-  DAD_LAUNCH(err, "gram_cholesky", (gram_cholesky_kernel<T>), dim3((unsigned)chunks, (unsigned)S), 256, smem1, st, G, r, h, chunks, pass,
-             tol, gram_partial, gram, tratio, dead, counters, status);
-  DAD_LAUNCH(err, "tri_solve", (tri_solve_kernel<T>), dim3((unsigned)ceil_div(h, 128), (unsigned)S), 128, smem2, st, G, r, h, gram,
-             dead, out32, planes, plane_rows);
+  DAD_LAUNCH(err, "gram_cholesky", (gram_cholesky_kernel<T>), dim3((unsigned)chunks, (unsigned)S), 256, smem1, st, G, r,
+             h, chunks, pass, tol, gram_partial, gram, tratio, dead, need2, counters, status);
+  DAD_LAUNCH(err, "tri_solve", (tri_solve_kernel<T>), dim3((unsigned)ceil_div(h, 128), (unsigned)S), 128, smem2, st, G, r,
+             h, pass, gram, dead, need2, out32, planes, plane_rows);
   return err;
 }
 template cudaError_t cholqr_pass<float>(float*, int, int, int64_t, int, double, double*, double*, double*,
-                                        unsigned char*, unsigned*, int*, float*, __nv_bfloat16*, int, cudaStream_t);
+                                        unsigned char*, int*, unsigned*, int*, float*, __nv_bfloat16*, int,
+                                        cudaStream_t);
 template cudaError_t cholqr_pass<double>(double*, int, int, int64_t, int, double, double*, double*, double*,
-                                         unsigned char*, unsigned*, int*, float*, __nv_bfloat16*, int, cudaStream_t);
+                                         unsigned char*, int*, unsigned*, int*, float*, __nv_bfloat16*, int,
+                                         cudaStream_t);
 
 }  // namespace dad
