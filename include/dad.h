@@ -162,6 +162,28 @@ dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* 
                            float* grad, dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Reconstruction without caller scratch (the paper has no counterpart: this is a packaging of
+ * dad_reconstruct for hosts that cannot allocate).  Same arguments, results and errors as
+ * dad_reconstruct, minus `ws`: the scratch is a fixed array of DAD_STATIC_SCRATCH_BYTES inside the
+ * library's device image, present on every GPU that loads the library for the life of the process.
+ * It is meant for callers that must not (or cannot) obtain device memory themselves -- a plug-in
+ * living inside another program's memory pool, a step running under a fixed device-memory budget,
+ * code that cannot afford the device-wide synchronisation an allocation implies.  The call makes no
+ * cudaMalloc/cudaFree and calls no allocating library routine.
+ *   - Problems whose scratch need (dad_reconstruct_workspace_bytes) exceeds
+ *     DAD_STATIC_SCRATCH_BYTES are refused with DAD_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device resolves the array's device address (and clears its status
+ *     words on `cuda_stream`); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     library clears what has to start at zero.  Two calls that overlap in time on the same GPU
+ *     (different streams, different host threads) race on it: serialise them, or use dad_reconstruct
+ *     with separate workspaces.  Device-side status is not reported for this entry point.
+ */
+#define DAD_STATIC_SCRATCH_BYTES (32u << 20)
+dad_status dad_reconstruct_static(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat,
+                                  float* grad, dad_dtype math, void* cuda_stream);
+
+/*
  * Device-side status of the work that used `ws`: synchronises `cuda_stream`, reads the status
  * words at the head of the workspace -- one written by the last dad_rank_compress on it, one by
  * the last dad_full_grad / dad_reconstruct on it -- and returns the first that is not DAD_OK

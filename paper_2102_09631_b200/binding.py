@@ -24,6 +24,7 @@ STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD
 # every symbol include/dad.h declares
 EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
            "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
+           "dad_reconstruct_static",
            "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.dad_reconstruct.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, ctypes.c_int, vp,
                                       ctypes.c_size_t, vp]
         L.dad_reconstruct.restype = ctypes.c_int
+        L.dad_reconstruct_static.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, ctypes.c_int, vp]
+        L.dad_reconstruct_static.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -179,6 +182,16 @@ def dad_reconstruct(h_in: int, h_out: int, K: int, Pcat, Qcat, grad, math: int =
     st = lib().dad_reconstruct(h_in, h_out, K, _ptr(Pcat), _ptr(Qcat), _ptr(grad), math, _ptr(ws),
                                ws.numel() if ws is not None else 0, _stream(stream))
     _check(st, "dad_reconstruct")
+
+
+DAD_STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def dad_reconstruct_static(h_in: int, h_out: int, K: int, Pcat, Qcat, grad, math: int = DAD_F32, stream=None):
+    """dad_reconstruct for callers that cannot provide scratch: the library's own fixed device array
+    (DAD_STATIC_SCRATCH_BYTES, shared by all calls on the device) stands in for `ws`."""
+    st = lib().dad_reconstruct_static(h_in, h_out, K, _ptr(Pcat), _ptr(Qcat), _ptr(grad), math, _stream(stream))
+    _check(st, "dad_reconstruct_static")
 
 
 def dad_check(ws, stream=None):
