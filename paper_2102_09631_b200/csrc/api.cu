@@ -97,13 +97,14 @@ GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_ope
   size_t off = 0;
   w.status = off;
   off += 256;
-  const size_t tiles = (size_t)(ceil_div(hx, 128) * ceil_div(hy, 128));
+  const int bn = umma_gemm_bn(hy);
+  const size_t tiles = (size_t)(ceil_div(hx, 128) * ceil_div(hy, bn));
   const int splits = umma_gemm_splits(hx, hy, ceil_div(N, 64) * S);
   w.n_counters = tiles;
   w.counters = off;
   off = align_up(off + tiles * sizeof(unsigned), 256);
   w.partial = off;
-  off = align_up(off + (splits > 1 ? tiles * (size_t)splits * 128 * 128 * 4 : 0), 256);
+  off = align_up(off + (splits > 1 ? tiles * (size_t)splits * 128 * (size_t)bn * 4 : 0), 256);
   w.Xb = w.Yb = off;
   if (convert_operands) {
     w.Xb = off;
@@ -161,6 +162,12 @@ static cudaError_t run_compress(const dad_layer& L, const void* A, const void* D
     DAD_STEP(cols_acc<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, Y, r, G, nullptr, part, ctr_cols, st));  // Gt = W^T D
     // the second pass returns at once for sites whose first pass was well conditioned, so both write the outputs
     float* q32 = (f64 && k == iters - 1) ? Q : nullptr;
+    if constexpr (!f64) {
+      if (orth_cluster_fits(r, ho)) {
+        DAD_STEP(orth_cluster(reinterpret_cast<float*>(G), S, r, ho, tol, status, nullptr, nullptr, 0, st));
+        continue;
+      }
+    }
     DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,
                                nullptr, 0, st));
     DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,
@@ -214,10 +221,14 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
     DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, nullptr, nullptr, Fz, hi, part, ctr_cols, status, st));     // Z = Y^T A
     DAD_STEP(umma_rows_dot(tmA_rows, tmFz, S, N, hi, r, Yt, w.Npad, status, st));                                  // W = A Z^T
     DAD_STEP(umma_cols_acc(tmD_cols, tmYt, S, N, ho, r, Q, nullptr, nullptr, 0, part, ctr_cols, status, st));       // Gt = W^T D
-    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, nullptr,
-                                Fq, rp, st));
-    DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, nullptr,
-                                Fq, rp, st));
+    if (orth_cluster_fits(r, ho)) {
+      DAD_STEP(orth_cluster(Q, S, r, ho, tol, status, nullptr, Fq, rp, st));
+    } else {
+      DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status,
+                                  nullptr, Fq, rp, st));
+      DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status,
+                                  nullptr, Fq, rp, st));
+    }
   }
   DAD_STEP(umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st));
   DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, P, nullptr, nullptr, 0, part, ctr_cols, status, st));

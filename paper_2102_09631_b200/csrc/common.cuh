@@ -101,6 +101,12 @@ cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, dou
                         double* gram, double* tratio, unsigned char* dead, int* need2, unsigned* counters,
                         int* status, float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
 
+// The same orthonormalisation (both passes, second one decided on the device) in one launch, for
+// fp32 storage: a thread-block cluster per site keeps the vectors in shared memory throughout.
+bool orth_cluster_fits(int r, int64_t h);
+cudaError_t orth_cluster(float* G, int S, int r, int64_t h, double tol, int* status, float* out32,
+                         __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
+
 // C[a][b] = sum_{s,n} X[s][n][a] * Y[s][n][b]  (fp32 FMA), C: hx x hy fp32 contiguous
 cudaError_t gemm_tn_simt(dad_dtype dt, const void* X, int64_t ldX, int64_t strideX, const void* Y,
                          int64_t ldY, int64_t strideY, int S, int64_t N, int64_t hx, int64_t hy, float* C,
@@ -122,6 +128,7 @@ bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t
                        uint64_t s2_bytes, uint32_t box0, uint32_t box1);
 int umma_rank_pad(int r);
 int umma_cols_acc_splits(int S, int64_t N, int64_t h);
+int umma_gemm_bn(int64_t hy);
 int umma_gemm_splits(int64_t hx, int64_t hy, int64_t k_blocks);
 cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S, int64_t N, int64_t h, int r,
                           __nv_bfloat16* yt_planes, int64_t ld_planes, int* status, cudaStream_t st);

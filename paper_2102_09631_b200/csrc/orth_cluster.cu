@@ -1,0 +1,317 @@
+// Orthonormalisation of the r iterate vectors of a site in ONE launch (fp32 storage pipeline):
+// a thread-block cluster of C CTAs per site, each holding a slab of r x W columns in shared
+// memory for the whole Cholesky-QR (both passes), so the vectors are read from and written to
+// global memory exactly once.
+//
+//   pass:  partial Gram of the slab (fp64, BS x BS register blocks)  ->  sum of the C partials
+//          over distributed shared memory, in rank order, by every CTA (all CTAs get the identical
+//          r x r matrix)  ->  Cholesky in shared memory (same pivot floor and zeroing rule as
+//          orth.cu)  ->  forward substitution down each column of the slab, in place, four rows
+//          at a time.
+//   A second pass runs when the first shows R_jj < 1e-3 ||g_j|| for some vector; the decision is
+//   identical in all CTAs of the cluster because they factor the same matrix.
+//
+// The substitution reads the already-solved vectors back in fp32; that perturbs the right-hand
+// side by one fp32 rounding, the same size as the rounding of the stored input itself.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace dad {
+
+namespace {
+constexpr double kPivotFloor = 1e-14;          // (1e-7)^2 of the squared length
+constexpr double kSecondPassBelowSq = 1e-6;    // (1e-3)^2: ratio of squared lengths that asks for a second pass
+constexpr int kThreads = 256;
+
+struct OrthGeom {
+  int rp;       // r rounded up to the register block (a multiple of 4)
+  int W;        // columns per CTA (multiple of 4)
+  int Wp;       // padded row length of the slab in floats
+  int nblocks;  // lower-triangular register blocks of the Gram matrix
+  int cgs;      // column groups the slab is split into for the Gram phase
+  size_t off_gram, off_L, off_vec, total;  // byte offsets after the slab
+};
+
+template <int BS>
+__host__ __device__ inline OrthGeom orth_geom(int r, int64_t h, int C) {
+  OrthGeom g;
+  constexpr int RB = BS < 4 ? 4 : BS;
+  g.rp = (r + RB - 1) / RB * RB;
+  int W = (int)((h + C - 1) / C);
+  g.W = (W + 3) / 4 * 4;
+  g.Wp = g.W + 2;  // even (float2 accesses), and rows 8 apart do not share a bank
+  const int nb = g.rp / BS;
+  g.nblocks = nb * (nb + 1) / 2;
+  g.cgs = kThreads / g.nblocks;
+  if (g.cgs < 1) g.cgs = 1;
+  if (g.cgs > 8) g.cgs = 8;
+  size_t off = sizeof(float) * (size_t)g.rp * g.Wp;
+  off = (off + 15) / 16 * 16;
+  g.off_gram = off;  // this CTA's partial Gram, rp x rp doubles (read by the other CTAs of the cluster)
+  off += sizeof(double) * (size_t)g.rp * g.rp;
+  g.off_L = off;  // rp x (rp + 1) doubles
+  off += sizeof(double) * (size_t)g.rp * (g.rp + 1);
+  g.off_vec = off;  // 3 x rp doubles: squared lengths, first-pass squared ratios, inverse diagonal
+  off += sizeof(double) * 3 * (size_t)g.rp;
+  g.total = off;
+  return g;
+}
+
+inline int cluster_size_for(int64_t h) {
+  int C = 1;
+  while (C < 8 && h / (C * 2) >= 128) C *= 2;
+  return C;
+}
+}  // namespace
+
+template <int BS>
+__global__ void __launch_bounds__(kThreads)
+orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, int* __restrict__ status,
+                    float* __restrict__ out32, __nv_bfloat16* __restrict__ planes, int plane_rows) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const OrthGeom g = orth_geom<BS>(r, h, C);
+  float* slab = reinterpret_cast<float*>(smem_raw);
+  double* gram = reinterpret_cast<double*>(smem_raw + g.off_gram);
+  double* Lm = reinterpret_cast<double*>(smem_raw + g.off_L);
+  double* diag0 = reinterpret_cast<double*>(smem_raw + g.off_vec);
+  double* ratio1sq = diag0 + g.rp;
+  double* inv_l = ratio1sq + g.rp;
+  __shared__ int need2_s;
+  __shared__ unsigned char dead_row[DAD_MAX_RANK];
+
+  const int tid = threadIdx.x;
+  const int s = blockIdx.y;
+  const int rank = (int)cluster.block_rank();
+  const int rp = g.rp, W = g.W, Wp = g.Wp, LR = rp + 1;
+  const int64_t c0 = (int64_t)rank * W;
+  float* Gs = G + (int64_t)s * r * h;
+  const double tol2 = tol * tol;
+
+  // ---- load the slab (rows >= r and columns >= h are zero) ----
+  for (int idx = tid; idx < rp * W; idx += kThreads) {
+    const int j = idx / W, c = idx % W;
+    slab[j * Wp + c] = (j < r && c0 + c < h) ? Gs[(int64_t)j * h + c0 + c] : 0.f;
+  }
+  if (tid < DAD_MAX_RANK) dead_row[tid] = 0;
+  __syncthreads();
+
+  for (int pass = 0; pass < 2; ++pass) {
+    // ---- partial Gram of the slab: BS x BS register blocks of the lower triangle, fp64.  The slab is cut
+    //      into column groups; the groups add their blocks into `gram` one after the other (fixed order). ----
+    {
+      const int Wc = ((W + g.cgs - 1) / g.cgs + 3) / 4 * 4;
+      const int item = tid;
+      const bool active = item < g.nblocks * g.cgs;  // nblocks * cgs <= kThreads by construction, or cgs == 1
+      const int rounds = (g.nblocks + kThreads - 1) / kThreads;  // > 1 only when cgs == 1
+      for (int round = 0; round < rounds; ++round) {
+        const int b = (g.cgs > 1) ? item % g.nblocks : item + round * kThreads;
+        const int grp = (g.cgs > 1) ? item / g.nblocks : 0;
+        const bool mine = (g.cgs > 1) ? active : b < g.nblocks;
+        int bi = 0, bj = 0;
+        double acc[BS][BS];
+#pragma unroll
+        for (int u = 0; u < BS; ++u)
+#pragma unroll
+          for (int v = 0; v < BS; ++v) acc[u][v] = 0.0;
+        if (mine) {
+          while ((bi + 1) * (bi + 2) / 2 <= b) ++bi;  // block row: bi(bi+1)/2 <= b
+          bj = b - bi * (bi + 1) / 2;
+          const int cbeg = grp * Wc, cend = (cbeg + Wc < W) ? cbeg + Wc : W;
+          const float* ra = slab + (bi * BS) * Wp;
+          const float* rb = slab + (bj * BS) * Wp;
+          for (int c = cbeg; c < cend; ++c) {
+            double a[BS], bb[BS];
+#pragma unroll
+            for (int u = 0; u < BS; ++u) a[u] = (double)ra[u * Wp + c];
+#pragma unroll
+            for (int v = 0; v < BS; ++v) bb[v] = (double)rb[v * Wp + c];
+#pragma unroll
+            for (int u = 0; u < BS; ++u)
+#pragma unroll
+              for (int v = 0; v < BS; ++v) acc[u][v] += a[u] * bb[v];
+          }
+        }
+        for (int turn = 0; turn < g.cgs; ++turn) {
+          if (mine && grp == turn) {
+#pragma unroll
+            for (int u = 0; u < BS; ++u)
+#pragma unroll
+              for (int v = 0; v < BS; ++v) {
+                double* dst = gram + (bi * BS + u) * rp + bj * BS + v;
+                *dst = (turn == 0) ? acc[u][v] : *dst + acc[u][v];
+              }
+          }
+          __syncthreads();
+        }
+      }
+    }
+    // ---- sum the partials of all CTAs of the cluster, in rank order ----
+    cluster.sync();
+    for (int e = tid; e < rp * rp; e += kThreads) {
+      const int i = e / rp, j = e % rp;
+      if (j <= i) {
+        double t[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) t[q] = (q < C) ? cluster.map_shared_rank(gram, q)[e] : 0.0;
+        double v = t[0];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) v += t[q];
+        Lm[i * LR + j] = v;
+      }
+    }
+    cluster.sync();  // nobody rewrites its partial while a neighbour still reads it
+    if (tid < rp) diag0[tid] = Lm[tid * LR + tid];
+    if (tid == 0) need2_s = 0;
+    __syncthreads();
+
+    // ---- Cholesky, left-looking, one barrier per column: thread i owns row i; for column j it forms
+    //      c_ij = G_ij - sum_{l<j} L_il L_jl, and (redundantly, so that no second barrier is needed) the
+    //      pivot of row j, on which every thread takes the same decisions ----
+    for (int j = 0; j < rp; ++j) {
+      const int i = tid;
+      if (i >= j && i < rp) {
+        // the diagonal is read from its saved copy: thread j overwrites Lm[j][j] in this very step
+        double d = diag0[j], c = Lm[i * LR + j];
+        for (int l = 0; l < j; ++l) {
+          const double a = Lm[j * LR + l];
+          d -= a * a;
+          c -= Lm[i * LR + l] * a;
+        }
+        const double orig = diag0[j];
+        double piv = d;
+        int is_dead = 0, bad = 0;
+        if (!(orig == orig) || orig > 1.7e308) {
+          bad = 1;
+          is_dead = 1;
+        } else if (!(orig > 0.0)) {
+          is_dead = 1;
+        } else {
+          const double floor_ = kPivotFloor * orig;
+          if (!(piv > floor_)) piv = floor_;
+          if (pass == 1 && !(ratio1sq[j] * piv > tol2)) is_dead = 1;  // total remainder vs. the original length
+        }
+        if (is_dead) piv = 1.0;
+        const double l_jj = sqrt(piv);
+        if (i == j) {
+          if (bad && status) *status = (int)DAD_ERR_NUMERIC;
+          if (pass == 0) {
+            const double t2 = is_dead ? 0.0 : piv / orig;  // (R_jj / ||g_j||)^2
+            ratio1sq[j] = t2;
+            if (!is_dead && t2 < kSecondPassBelowSq) need2_s = 1;
+          }
+          if (is_dead) dead_row[j] = 1;
+          Lm[j * LR + j] = l_jj;
+          inv_l[j] = 1.0 / l_jj;
+        } else {
+          Lm[i * LR + j] = is_dead ? 0.0 : c / l_jj;
+        }
+      }
+      __syncthreads();
+    }
+
+    // ---- forward substitution down each column of the slab, in place: two adjacent columns per thread,
+    //      four rows at a time so that every solved value is read (and widened) once per row block ----
+    for (int c = 2 * tid; c < W; c += 2 * kThreads) {
+      for (int j0 = 0; j0 < rp; j0 += 4) {
+        double v[4][2];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float2 x = *reinterpret_cast<const float2*>(slab + (j0 + u) * Wp + c);
+          v[u][0] = (double)x.x;
+          v[u][1] = (double)x.y;
+        }
+        for (int l = 0; l < j0; ++l) {
+          const float2 q = *reinterpret_cast<const float2*>(slab + l * Wp + c);
+          const double q0 = (double)q.x, q1 = (double)q.y;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const double a = Lm[(j0 + u) * LR + l];
+            v[u][0] -= a * q0;
+            v[u][1] -= a * q1;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int j = j0 + u;
+          const double il = dead_row[j] ? 0.0 : inv_l[j];
+          // the value stored (and used by the rows below) is the fp32-rounded one
+          const float o0 = (float)(v[u][0] * il), o1 = (float)(v[u][1] * il);
+          *reinterpret_cast<float2*>(slab + j * Wp + c) = make_float2(o0, o1);
+#pragma unroll
+          for (int w = u + 1; w < 4; ++w) {
+            const double a = Lm[(j0 + w) * LR + j];
+            v[w][0] -= a * (double)o0;
+            v[w][1] -= a * (double)o1;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    if (need2_s == 0) break;  // same matrix, same decision in every CTA of the cluster
+  }
+
+  // ---- write the orthonormal vectors (and their bf16 hi/lo planes) ----
+  for (int idx = tid; idx < r * W; idx += kThreads) {
+    const int j = idx / W, c = idx % W;
+    if (c0 + c < h) {
+      const float f = slab[j * Wp + c];
+      const int64_t col = c0 + c;
+      Gs[(int64_t)j * h + col] = f;
+      if (out32) out32[((int64_t)s * r + j) * h + col] = f;
+      if (planes) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(f);
+        planes[(((int64_t)s * 2 + 0) * plane_rows + j) * h + col] = hi;
+        planes[(((int64_t)s * 2 + 1) * plane_rows + j) * h + col] = __float2bfloat16_rn(f - __bfloat162float(hi));
+      }
+    }
+  }
+}
+
+template <int BS>
+static cudaError_t launch_orth_cluster(float* G, int S, int r, int64_t h, int C, double tol, int* status, float* out32,
+                                       __nv_bfloat16* planes, int plane_rows, size_t smem, cudaStream_t st) {
+  auto kernel = orth_cluster_kernel<BS>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)C, (unsigned)S, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const bool timed = g_timing.load(std::memory_order_relaxed);
+  if (timed) timing_mark("orth_cluster", st, true);
+  err = cudaLaunchKernelEx(&cfg, kernel, G, r, h, C, tol, status, out32, planes, plane_rows);
+  if (timed) timing_mark("orth_cluster", st, false);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return err;
+}
+
+// Whether the one-launch kernel takes this shape (the slab of a CTA has to fit in shared memory).
+bool orth_cluster_fits(int r, int64_t h) {
+  if (h > (int64_t)1 << 30) return false;
+  const int C = cluster_size_for(h);
+  const size_t need = r >= 32 ? orth_geom<8>(r, h, C).total : orth_geom<2>(r, h, C).total;
+  return need <= 200 * 1024;
+}
+
+// Cholesky-QR (one or two passes, decided on the device) of the rows of G (S x r x h fp32, in place).
+cudaError_t orth_cluster(float* G, int S, int r, int64_t h, double tol, int* status, float* out32,
+                         __nv_bfloat16* planes, int plane_rows, cudaStream_t st) {
+  const int C = cluster_size_for(h);
+  if (r >= 32)
+    return launch_orth_cluster<8>(G, S, r, h, C, tol, status, out32, planes, plane_rows, orth_geom<8>(r, h, C).total, st);
+  return launch_orth_cluster<2>(G, S, r, h, C, tol, status, out32, planes, plane_rows, orth_geom<2>(r, h, C).total, st);
+}
+
+}  // namespace dad

@@ -383,8 +383,12 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
   }
 }
 
+// Tile width of the dense product: 256 columns keep the MMAs under the shared-memory read rate
+// (a 128 x 128 x 16 MMA needs 128 B/clk of operands, a 128 x 256 x 16 one 96 B/clk).
+int umma_gemm_bn(int64_t hy) { return hy > 128 ? 256 : 128; }
+
 int umma_gemm_splits(int64_t hx, int64_t hy, int64_t k_blocks) {
-  const int64_t tiles = ceil_div(hx, 128) * ceil_div(hy, 128);
+  const int64_t tiles = ceil_div(hx, 128) * ceil_div(hy, umma_gemm_bn(hy));
   int64_t splits = 148 / tiles;
   if (splits > k_blocks / 8) splits = k_blocks / 8;
   if (splits > 32) splits = 32;
@@ -408,7 +412,9 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, int S, 
   p.partial = partial;
   p.counters = counters;
   p.status = status;
-  dim3 grid((unsigned)ceil_div(hx, 128), (unsigned)(ceil_div(hy, 128) * p.splits), 1);
+  const int bn = umma_gemm_bn(hy);
+  dim3 grid((unsigned)ceil_div(hx, 128), (unsigned)(ceil_div(hy, bn) * p.splits), 1);
+  if (bn == 256) return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st);
   return launch_umma<128, true, true, 1, EPI_C, 6>(tmX, tmY, p, grid, "gemm_tn_tc", st);
 }
 
