@@ -40,6 +40,8 @@ def parse_args():
                     help="distinct transformer blocks of input data kept in HBM and cycled through")
     ap.add_argument("--blocks", type=int, default=None,
                     help="run only this many of the network's blocks per step (profiling captures); default all")
+    ap.add_argument("--no-group", action="store_true",
+                    help="one call per layer instead of stacking the same-shape layers of a block into one call")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -214,32 +216,35 @@ def run_ours(args):
     RB = max(1, min(cfg.blocks, args.resident_blocks))
 
     # inputs: RB distinct blocks of layers resident in HBM, cycled over the network's blocks
+    # call units: the layers of one shape inside a block (e.g. the four attention projections) are stacked as
+    # extra slices of one call -- sites and layers are independent in the power iterations -- unless --no-group
+    units = [(sh, 1) for sh in layers] if args.no_group else [(sh, sh.count) for sh in cfg.layers]
     data = []
     for b in range(RB):
         blk = []
-        for li, sh in enumerate(layers):
-            seed = wl.seed_for(cfg.index, b * len(layers) + li, rank)
+        for ui, (sh, groups) in enumerate(units):
+            seed = wl.seed_for(cfg.index, b * len(units) + ui, rank)
             if cfg.index == 1:
-                A, D = wl.gaussian_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+                A, D = wl.gaussian_layer(cfg.S * groups, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
             else:
-                A, D = wl.decaying_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
-            blk.append((A, D, wl.start_block(cfg.S, r, sh.h_out, seed, dev)))
+                A, D = wl.decaying_layer(cfg.S * groups, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+            blk.append((A, D, wl.start_block(cfg.S * groups, r, sh.h_out, seed, dev)))
         data.append(blk)
     plans = {}
-    for li, sh in enumerate(layers):
-        key = (sh.h_in, sh.h_out)
+    for ui, (sh, groups) in enumerate(units):
+        key = (sh.h_in, sh.h_out, groups)
         if key not in plans:
-            A, D, _ = data[0][li]
-            plans[key] = B.LayerPlan(A, D, r, iters)
+            A, D, _ = data[0][ui]
+            plans[key] = B.LayerPlan(A, D, r, iters, groups=groups)
     input_bytes = sum(A.numel() * A.element_size() + D.numel() * D.element_size() for blk in data for A, D, _ in blk)
     stream = torch.cuda.current_stream()
 
     def step():
         for b in range(cfg.blocks):
             blk = data[b % RB]
-            for li, sh in enumerate(layers):
-                A, D, Q0 = blk[li]
-                plans[(sh.h_in, sh.h_out)].step(A, D, Q0, stream)
+            for ui, (sh, groups) in enumerate(units):
+                A, D, Q0 = blk[ui]
+                plans[(sh.h_in, sh.h_out, groups)].step(A, D, Q0, stream)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -311,26 +316,26 @@ def run_ours(args):
     if not args.no_e2e:
         host = [(A.cpu().pin_memory(), D.cpu().pin_memory(), Q0.cpu().pin_memory()) for A, D, Q0 in data[0]]
         stage = {}
-        for li, sh in enumerate(layers):
-            key = (sh.h_in, sh.h_out)
+        for ui, (sh, groups) in enumerate(units):
+            key = (sh.h_in, sh.h_out, groups)
             if key not in stage:
-                A, D, Q0 = data[0][li]
+                A, D, Q0 = data[0][ui]
                 stage[key] = (torch.empty_like(A), torch.empty_like(D), torch.empty_like(Q0),
-                              torch.empty(sh.h_in, sh.h_out, dtype=torch.float32).pin_memory())
+                              torch.empty(groups, sh.h_in, sh.h_out, dtype=torch.float32).pin_memory())
         h2d = sum(a.numel() * a.element_size() + d.numel() * d.element_size() + q.numel() * 4 for a, d, q in host) * cfg.blocks
         d2h = sum(sh.h_in * sh.h_out * 4 for sh in layers) * cfg.blocks
 
         def e2e_step():
             for b in range(cfg.blocks):
-                for li, sh in enumerate(layers):
-                    key = (sh.h_in, sh.h_out)
+                for ui, (sh, groups) in enumerate(units):
+                    key = (sh.h_in, sh.h_out, groups)
                     As, Ds, Qs, gh = stage[key]
-                    a, d, q = host[li]
+                    a, d, q = host[ui]
                     As.copy_(a, non_blocking=True)
                     Ds.copy_(d, non_blocking=True)
                     Qs.copy_(q, non_blocking=True)
-                    grad = plans[key].step(As, Ds, Qs, stream)
-                    gh.copy_(grad, non_blocking=True)
+                    plans[key].step(As, Ds, Qs, stream)
+                    gh.copy_(plans[key].grads, non_blocking=True)
 
         e2e_step()
         sync_all()
@@ -362,6 +367,9 @@ def run_ours(args):
                 "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "bf16", "data": "synthetic",
                 "config": {"workload": workload_name(cfg, r, iters),
                            "l2": f"inputs larger than L2: {RB} resident block(s), {input_bytes / 1e9:.2f} GB, cycled",
+                           "calls": ("one call per layer" if args.no_group else
+                                     "same-shape layers of a block stacked as extra slices of one call: " +
+                                     ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
                 "kernels": kernels,

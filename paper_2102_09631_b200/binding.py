@@ -219,11 +219,20 @@ def bytes_array(S: int):
 
 class LayerPlan:
     """Buffers for one layer shape, allocated once: factors, stacks, gradient and workspace.
-    `step` runs compress -> gather -> reconstruct on the current stream (marshalling only)."""
+    `step` runs compress -> gather -> reconstruct on the current stream (marshalling only).
 
-    def __init__(self, A: torch.Tensor, D: torch.Tensor, r: int, iters: int, zero_copy_gather: bool = False):
+    `groups` > 1 stacks that many layers of the same shape in one plan: A and D then hold
+    groups * S slices (layer g owns slices g*S .. g*S+S-1), the power iterations of all of them run
+    in the same launches (slices are independent), and each layer is reconstructed from its own rows
+    of the stacks; `grad` is then groups x h_in x h_out."""
+
+    def __init__(self, A: torch.Tensor, D: torch.Tensor, r: int, iters: int, zero_copy_gather: bool = False,
+                 groups: int = 1):
         self.layer = make_layer(A, D)
         L = self.layer
+        if groups < 1 or L.S % groups:
+            raise ValueError("the slice count must be a multiple of `groups`")
+        self.groups, self.sites = groups, L.S // groups
         dev = A.device
         self.r, self.iters = r, iters
         self.P = torch.empty(L.S, r, L.h_in, device=dev, dtype=torch.float32)
@@ -234,17 +243,22 @@ class LayerPlan:
         else:
             self.Pcat = torch.empty(L.S * r, L.h_in, device=dev, dtype=torch.float32)
             self.Qcat = torch.empty(L.S * r, L.h_out, device=dev, dtype=torch.float32)
-        self.grad = torch.empty(L.h_in, L.h_out, device=dev, dtype=torch.float32)
+        self.grads = torch.empty(groups, L.h_in, L.h_out, device=dev, dtype=torch.float32)
+        self.grad = self.grads[0] if groups == 1 else self.grads
         self.math = L.dtype
         nws = dad_workspace_bytes(L, r, iters)
         if nws == 0:
             raise ValueError("invalid layer / rank / iteration count")
-        self.ws = new_workspace(max(nws, dad_reconstruct_workspace_bytes(L.h_in, L.h_out, L.S * r, self.math)), dev)
+        self.K = self.sites * r
+        self.ws = new_workspace(max(nws, dad_reconstruct_workspace_bytes(L.h_in, L.h_out, self.K, self.math)), dev)
         self.bytes_tx = bytes_array(L.S)
 
     def step(self, A, D, Q0, stream=None):
         L = self.layer
         dad_rank_compress(L, A, D, self.r, self.iters, Q0, self.P, self.Q, self.sigma, self.ws, stream)
         dad_gather_factors(L, self.r, self.P, self.Q, self.Pcat, self.Qcat, self.bytes_tx, stream)
-        dad_reconstruct(L.h_in, L.h_out, L.S * self.r, self.Pcat, self.Qcat, self.grad, self.math, self.ws, stream)
+        for g in range(self.groups):
+            rows = slice(g * self.K, (g + 1) * self.K)
+            dad_reconstruct(L.h_in, L.h_out, self.K, self.Pcat[rows], self.Qcat[rows], self.grads[g], self.math,
+                            self.ws, stream)
         return self.grad

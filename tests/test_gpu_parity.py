@@ -248,3 +248,26 @@ def test_compress_at_full_size_on_sampled_sites(oracle, B):
         Qg = plan.Q[s].double().cpu().numpy()
         assert np.linalg.norm(Qg @ Qg.T - np.eye(cfg.r)) <= 1e-3
     assert list(plan.bytes_tx) == [oracle.bytes_rank(cfg.r, shape.h_in, shape.h_out)] * cfg.S
+
+
+def test_stacked_layers_match_separate_calls(oracle, B):
+    """Several layers of one shape stacked as extra slices of one call (groups > 1) give, layer by layer,
+    what separate calls give -- bit for bit -- and agree with the oracle."""
+    dev = torch.device("cuda:0")
+    S, groups, N, h_in, h_out, r, iters = 3, 2, 200, 128, 192, 8, 2
+    A, D = wl.decaying_layer(S * groups, N, h_in, h_out, 77, torch.bfloat16)
+    Q0 = wl.start_block(S * groups, r, h_out, 77)
+    Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
+    plan = B.LayerPlan(Ad, Dd, r, iters, groups=groups)
+    grads = plan.step(Ad, Dd, Q0d).clone()
+    B.dad_check(plan.ws)
+    assert grads.shape == (groups, h_in, h_out)
+    for g in range(groups):
+        sl = slice(g * S, (g + 1) * S)
+        single = B.LayerPlan(Ad[sl], Dd[sl], r, iters)
+        single.step(Ad[sl], Dd[sl], Q0d[sl])
+        B.dad_check(single.ws)
+        assert torch.equal(single.grad, grads[g])
+        ref = oracle.rank_dad_layer(A[sl], D[sl], Q0[sl], iters)
+        assert rel(grads[g].double().cpu().numpy(), ref["grad"]) <= TOL[torch.bfloat16]
+    assert list(plan.bytes_tx) == [oracle.bytes_rank(r, h_in, h_out)] * (S * groups)
