@@ -91,6 +91,9 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   float* Gs = G + (int64_t)s * r * h;
   const double tol2 = tol * tol;
 
+  // the next kernel in the stream may begin its set-up now; it waits for this grid before touching memory
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   // ---- load the slab (rows >= r and columns >= h are zero) ----
   for (int idx = tid; idx < rp * W; idx += kThreads) {
     const int j = idx / W, c = idx % W;

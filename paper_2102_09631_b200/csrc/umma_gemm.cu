@@ -92,6 +92,13 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t tmem_base = tmem_base_s;
   volatile int* abortp = &abort_flag;
 
+  // Programmatic dependent launch: everything above touched only this CTA's own shared and tensor
+  // memory, so it may overlap the tail of the previous kernel in the stream.  From here on the kernel
+  // reads what earlier kernels wrote (and overwrites what they read): wait for them to finish.  The
+  // next kernel in the stream is allowed to start its own set-up right away.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   if (warp == 0) {
     if (lane == 0) {
       prefetch_tmap(&tmA);
@@ -330,7 +337,21 @@ static cudaError_t launch_umma(const CUtensorMap& tmA, const CUtensorMap& tmB, c
   auto kernel = umma_kernel<BN, A_MN, B_MN, TERMS, EPI, STAGES>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  DAD_LAUNCH(err, tag, kernel, grid, 192, smem, st, tmA, tmB, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(192, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernel
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const bool timed = g_timing.load(std::memory_order_relaxed);
+  if (timed) timing_mark(tag, st, true);
+  err = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+  if (timed) timing_mark(tag, st, false);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
   return err;
 }
 
