@@ -46,6 +46,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile-pass", action="store_true")
+    ap.add_argument("--no-full-grad", action="store_true", help="skip timing the uncompressed dAD gradient")
     return ap.parse_args()
 
 
@@ -192,17 +193,14 @@ def run_reference(args):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2102_09631_b200 import binding as B, build as dad_build, workloads as wl
+    from paper_2102_09631_b200 import binding as B, build as dad_build, multi, workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = multi.env_rank_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    multi.init("nccl", dev)
     dad_build.build()
     B.lib()
 
@@ -249,7 +247,7 @@ def run_ours(args):
     def sync_all():
         torch.cuda.synchronize()
         if world > 1:
-            dist.barrier()
+            multi.barrier()
             torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -270,14 +268,10 @@ def run_ours(args):
     sync_all()
     launches = B.dad_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = multi.max_over_ranks(ev0.elapsed_time(ev1), dev)
     ms_per_step = ms / args.steps
     n_layers = cfg.n_layers()
-    value = world * n_layers / (ms_per_step * 1e-3)
+    value = multi.whole_job_rate(n_layers, world, ms_per_step * 1e-3)
 
     # ---- per-kernel times: a second pass of the same steps with events around every launch ----
     peaks = read_peaks()
@@ -310,6 +304,38 @@ def run_ours(args):
         else:
             roofline = {"bound": "hbm", "kernel": name, "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": None, "traffic": None, "peak_source": peaks["source"]}
+
+    # ---- the uncompressed dAD gradient (sum_s A_s^T D_s) of each layer shape: the tensor-bound product ----
+    full_grad = None
+    if not args.no_full_grad:
+        rows = []
+        flops_total, ms_total = 0.0, 0.0
+        for ui, (sh, groups) in enumerate(units):
+            A, D, _ = data[0][ui]
+            A1, D1 = A[:cfg.S], D[:cfg.S]          # one layer's slices
+            L1 = B.make_layer(A1, D1)
+            g = torch.empty(sh.h_in, sh.h_out, device=dev, dtype=torch.float32)
+            ws = B.new_workspace(B.dad_workspace_bytes(L1, 1, 0), dev)
+            for _ in range(2):
+                B.dad_full_grad(L1, A1, D1, g, None, ws, stream)
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = 5
+            torch.cuda.synchronize()
+            f0.record(stream)
+            for _ in range(reps):
+                B.dad_full_grad(L1, A1, D1, g, None, ws, stream)
+            f1.record(stream)
+            torch.cuda.synchronize()
+            B.dad_check(ws)
+            t_ms = f0.elapsed_time(f1) / reps
+            fl = 2.0 * cfg.S * cfg.N * sh.h_in * sh.h_out
+            flops_total += fl * sh.count
+            ms_total += t_ms * sh.count
+            rows.append({"layer": f"{sh.h_in}->{sh.h_out}", "us": t_ms * 1e3, "tflops": fl / (t_ms * 1e-3) / 1e12})
+        tf = flops_total / (ms_total * 1e-3) / 1e12
+        full_grad = {"bound": "tensor" if cfg.dtype == "bf16" else "alu", "achieved": tf, "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
+                     "layers_per_s": sum(sh.count for sh in cfg.layers) / (ms_total * 1e-3), "per_shape": rows}
 
     # ---- end to end: inputs start in pinned host memory, the gradient ends there ------------------
     e2e = None
@@ -345,21 +371,23 @@ def run_ours(args):
             e2e_step()
         e1.record(stream)
         sync_all()
-        ems = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ems], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
-        e2e = {"value": world * n_layers * args.e2e_steps / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        ems = multi.max_over_ranks(e0.elapsed_time(e1), dev)
+        e2e = {"value": multi.whole_job_rate(n_layers * args.e2e_steps, world, ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import dad_oracle
         dad_oracle.build()
-        lps, secs, sample = oracle_sample(cfg, r, iters)
-        cpu = {"value": lps, "unit": UNIT, "cores": min(dad_oracle.max_threads(), cfg.S), "kind": "oracle",
-               "sample": sample, "seconds": secs}
+        # repeat the sample until about ten seconds of oracle time have gone by (at most 8 times)
+        inv, secs, reps, sample = 0.0, 0.0, 0, ""
+        while reps < 8 and (secs < 10.0 or reps == 0):
+            lps, s1, sample = oracle_sample(cfg, r, iters)
+            inv += 1.0 / lps
+            secs += s1
+            reps += 1
+        cpu = {"value": reps / inv, "unit": UNIT, "cores": min(dad_oracle.max_threads(), cfg.S), "kind": "oracle",
+               "sample": f"{reps}x [{sample}]", "seconds": secs}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -372,7 +400,7 @@ def run_ours(args):
                                      ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-                "kernels": kernels,
+                "kernels": kernels, "dad_full_grad": full_grad,
                 "stream_gbs": sum(sum(v for k, v in stream_bytes_per_layer(cfg, sh, iters).items() if not k.endswith("launches"))
                                   for sh in layers) * cfg.blocks / (ms_per_step * 1e-3) / 1e9}
         print(json.dumps(line))
