@@ -40,6 +40,8 @@ def parse_args():
                     help="distinct transformer blocks of input data kept in HBM and cycled through")
     ap.add_argument("--blocks", type=int, default=None,
                     help="run only this many of the network's blocks per step (profiling captures); default all")
+    ap.add_argument("--group-blocks", type=int, default=4,
+                    help="stack the same-shape layers of this many consecutive blocks into one call")
     ap.add_argument("--no-group", action="store_true",
                     help="one call per layer instead of stacking the same-shape layers of a block into one call")
     ap.add_argument("--e2e-steps", type=int, default=1)
@@ -211,12 +213,15 @@ def run_ours(args):
     r = args.rank or cfg.r
     iters = cfg.iters if args.iters is None else args.iters
     layers = expand_layers(cfg)
-    RB = max(1, min(cfg.blocks, args.resident_blocks))
-
-    # inputs: RB distinct blocks of layers resident in HBM, cycled over the network's blocks
-    # call units: the layers of one shape inside a block (e.g. the four attention projections) are stacked as
-    # extra slices of one call -- sites and layers are independent in the power iterations -- unless --no-group
-    units = [(sh, 1) for sh in layers] if args.no_group else [(sh, sh.count) for sh in cfg.layers]
+    # call units: after a backward pass every layer's (A, Delta) is at hand, and sites and layers are independent
+    # in the power iterations, so the layers of one shape from G consecutive blocks (e.g. 4 x 4 attention
+    # projections) are stacked as extra slices of one call -- unless --no-group (one call per layer)
+    G = 1
+    if not args.no_group:
+        G = max(g for g in range(1, max(1, args.group_blocks) + 1) if cfg.blocks % g == 0)
+    n_super = cfg.blocks // G                      # calls of each unit per step
+    RB = max(1, min(n_super, args.resident_blocks // G))   # distinct input sets resident in HBM, cycled
+    units = [(sh, 1) for sh in layers] if args.no_group else [(sh, sh.count * G) for sh in cfg.layers]
     data = []
     for b in range(RB):
         blk = []
@@ -238,7 +243,7 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     def step():
-        for b in range(cfg.blocks):
+        for b in range(n_super):
             blk = data[b % RB]
             for ui, (sh, groups) in enumerate(units):
                 A, D, Q0 = blk[ui]
@@ -348,11 +353,11 @@ def run_ours(args):
                 A, D, Q0 = data[0][ui]
                 stage[key] = (torch.empty_like(A), torch.empty_like(D), torch.empty_like(Q0),
                               torch.empty(groups, sh.h_in, sh.h_out, dtype=torch.float32).pin_memory())
-        h2d = sum(a.numel() * a.element_size() + d.numel() * d.element_size() + q.numel() * 4 for a, d, q in host) * cfg.blocks
+        h2d = sum(a.numel() * a.element_size() + d.numel() * d.element_size() + q.numel() * 4 for a, d, q in host) * n_super
         d2h = sum(sh.h_in * sh.h_out * 4 for sh in layers) * cfg.blocks
 
         def e2e_step():
-            for b in range(cfg.blocks):
+            for b in range(n_super):
                 for ui, (sh, groups) in enumerate(units):
                     key = (sh.h_in, sh.h_out, groups)
                     As, Ds, Qs, gh = stage[key]
@@ -394,9 +399,9 @@ def run_ours(args):
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "bf16", "data": "synthetic",
                 "config": {"workload": workload_name(cfg, r, iters),
-                           "l2": f"inputs larger than L2: {RB} resident block(s), {input_bytes / 1e9:.2f} GB, cycled",
+                           "l2": f"inputs larger than L2: {RB} resident input set(s) of {G} block(s), {input_bytes / 1e9:.2f} GB, cycled",
                            "calls": ("one call per layer" if args.no_group else
-                                     "same-shape layers of a block stacked as extra slices of one call: " +
+                                     f"same-shape layers of {G} consecutive block(s) stacked as extra slices of one call: " +
                                      ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
