@@ -8,8 +8,9 @@
 //          r x r matrix)  ->  Cholesky in shared memory (same pivot floor and zeroing rule as
 //          orth.cu)  ->  forward substitution down each column of the slab, in place, four rows
 //          at a time.
-//   A second pass runs when the first shows R_jj < 1e-3 ||g_j|| for some vector; the decision is
-//   identical in all CTAs of the cluster because they factor the same matrix.
+//   A second pass runs when the first shows R_jj < 1e-5 ||g_j|| for some vector (one fp64 pass leaves
+//   an orthogonality defect of about 1e-16 cond^2 <= 1e-6, the level of the fp32 storage itself); the
+//   decision is identical in all CTAs of the cluster because they factor the same matrix.
 //
 // The substitution reads the already-solved vectors back in fp32; that perturbs the right-hand
 // side by one fp32 rounding, the same size as the rounding of the stored input itself.
@@ -23,7 +24,7 @@ namespace dad {
 
 namespace {
 constexpr double kPivotFloor = 1e-14;          // (1e-7)^2 of the squared length
-constexpr double kSecondPassBelowSq = 1e-6;    // (1e-3)^2: ratio of squared lengths that asks for a second pass
+constexpr double kSecondPassBelowSq = 1e-10;   // (1e-5)^2: ratio of squared lengths that asks for a second pass
 constexpr int kThreads = 256;
 
 struct OrthGeom {
@@ -54,8 +55,8 @@ __host__ __device__ inline OrthGeom orth_geom(int r, int64_t h, int C) {
   off += sizeof(double) * (size_t)g.rp * g.rp;
   g.off_L = off;  // rp x (rp + 1) doubles
   off += sizeof(double) * (size_t)g.rp * (g.rp + 1);
-  g.off_vec = off;  // 3 x rp doubles: squared lengths, first-pass squared ratios, inverse diagonal
-  off += sizeof(double) * 3 * (size_t)g.rp;
+  g.off_vec = off;  // 4 x rp doubles: squared lengths, first-pass pivots, inverse diagonal, first-pass lengths
+  off += sizeof(double) * 4 * (size_t)g.rp;
   g.total = off;
   return g;
 }
@@ -78,8 +79,9 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   double* gram = reinterpret_cast<double*>(smem_raw + g.off_gram);
   double* Lm = reinterpret_cast<double*>(smem_raw + g.off_L);
   double* diag0 = reinterpret_cast<double*>(smem_raw + g.off_vec);
-  double* ratio1sq = diag0 + g.rp;
-  double* inv_l = ratio1sq + g.rp;
+  double* piv1 = diag0 + g.rp;   // first-pass pivots (squared R_jj)
+  double* inv_l = piv1 + g.rp;
+  double* orig1 = inv_l + g.rp;  // squared lengths before the first pass
   __shared__ int need2_s;
   __shared__ unsigned char dead_row[DAD_MAX_RANK];
 
@@ -95,9 +97,44 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // ---- load the slab (rows >= r and columns >= h are zero) ----
-  for (int idx = tid; idx < rp * W; idx += kThreads) {
-    const int j = idx / W, c = idx % W;
-    slab[j * Wp + c] = (j < r && c0 + c < h) ? Gs[(int64_t)j * h + c0 + c] : 0.f;
+  // Loads are issued eight at a time per thread before any is stored, so that their latencies overlap.
+  if ((h & 3) == 0) {
+    const int W4 = W / 4, total = rp * W4;
+    for (int base = 0; base < total; base += kThreads * 8) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = base + u * kThreads + tid;
+        const int j = idx / W4, c = (idx % W4) * 4;
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (idx < total && j < r && c0 + c < h) v[u] = *reinterpret_cast<const float4*>(Gs + (int64_t)j * h + c0 + c);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = base + u * kThreads + tid;
+        if (idx < total) {
+          float* dst = slab + (idx / W4) * Wp + (idx % W4) * 4;  // 8-byte aligned (Wp is even)
+          *reinterpret_cast<float2*>(dst) = make_float2(v[u].x, v[u].y);
+          *reinterpret_cast<float2*>(dst + 2) = make_float2(v[u].z, v[u].w);
+        }
+      }
+    }
+  } else {
+    const int total = rp * W;
+    for (int base = 0; base < total; base += kThreads * 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = base + u * kThreads + tid;
+        const int j = idx / W, c = idx % W;
+        v[u] = (idx < total && j < r && c0 + c < h) ? Gs[(int64_t)j * h + c0 + c] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = base + u * kThreads + tid;
+        if (idx < total) slab[(idx / W) * Wp + idx % W] = v[u];
+      }
+    }
   }
   if (tid < DAD_MAX_RANK) dead_row[tid] = 0;
   __syncthreads();
@@ -195,22 +232,23 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
         } else {
           const double floor_ = kPivotFloor * orig;
           if (!(piv > floor_)) piv = floor_;
-          if (pass == 1 && !(ratio1sq[j] * piv > tol2)) is_dead = 1;  // total remainder vs. the original length
+          // second pass: total remainder (R1_jj R2_jj)^2 against tol^2 of the squared length before pass one
+          if (pass == 1 && !(piv1[j] * piv > tol2 * orig1[j])) is_dead = 1;
         }
         if (is_dead) piv = 1.0;
-        const double l_jj = sqrt(piv);
+        const double il = rsqrt(piv);  // one reciprocal square root instead of a square root and divisions
         if (i == j) {
           if (bad && status) *status = (int)DAD_ERR_NUMERIC;
           if (pass == 0) {
-            const double t2 = is_dead ? 0.0 : piv / orig;  // (R_jj / ||g_j||)^2
-            ratio1sq[j] = t2;
-            if (!is_dead && t2 < kSecondPassBelowSq) need2_s = 1;
+            piv1[j] = is_dead ? 0.0 : piv;
+            orig1[j] = orig;
+            if (!is_dead && piv < kSecondPassBelowSq * orig) need2_s = 1;
           }
           if (is_dead) dead_row[j] = 1;
-          Lm[j * LR + j] = l_jj;
-          inv_l[j] = 1.0 / l_jj;
+          Lm[j * LR + j] = piv * il;
+          inv_l[j] = il;
         } else {
-          Lm[i * LR + j] = is_dead ? 0.0 : c / l_jj;
+          Lm[i * LR + j] = is_dead ? 0.0 : c * il;
         }
       }
       __syncthreads();
@@ -258,17 +296,44 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   }
 
   // ---- write the orthonormal vectors (and their bf16 hi/lo planes) ----
-  for (int idx = tid; idx < r * W; idx += kThreads) {
-    const int j = idx / W, c = idx % W;
-    if (c0 + c < h) {
-      const float f = slab[j * Wp + c];
+  if ((h & 3) == 0) {
+    const int W4 = W / 4;
+    for (int idx = tid; idx < r * W4; idx += kThreads) {
+      const int j = idx / W4, c = (idx % W4) * 4;
       const int64_t col = c0 + c;
-      Gs[(int64_t)j * h + col] = f;
-      if (out32) out32[((int64_t)s * r + j) * h + col] = f;
-      if (planes) {
-        const __nv_bfloat16 hi = __float2bfloat16_rn(f);
-        planes[(((int64_t)s * 2 + 0) * plane_rows + j) * h + col] = hi;
-        planes[(((int64_t)s * 2 + 1) * plane_rows + j) * h + col] = __float2bfloat16_rn(f - __bfloat162float(hi));
+      if (col < h) {
+        const float2 lo2 = *reinterpret_cast<const float2*>(slab + j * Wp + c);
+        const float2 hi2 = *reinterpret_cast<const float2*>(slab + j * Wp + c + 2);
+        const float f[4] = {lo2.x, lo2.y, hi2.x, hi2.y};
+        *reinterpret_cast<float4*>(Gs + (int64_t)j * h + col) = make_float4(f[0], f[1], f[2], f[3]);
+        if (out32) *reinterpret_cast<float4*>(out32 + ((int64_t)s * r + j) * h + col) = make_float4(f[0], f[1], f[2], f[3]);
+        if (planes) {
+          __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            hi[u] = __float2bfloat16_rn(f[u]);
+            lo[u] = __float2bfloat16_rn(f[u] - __bfloat162float(hi[u]));
+          }
+          __nv_bfloat16* ph = planes + (((int64_t)s * 2 + 0) * plane_rows + j) * h + col;  // 8-byte aligned
+          __nv_bfloat16* pl = planes + (((int64_t)s * 2 + 1) * plane_rows + j) * h + col;
+          *reinterpret_cast<uint2*>(ph) = *reinterpret_cast<const uint2*>(hi);
+          *reinterpret_cast<uint2*>(pl) = *reinterpret_cast<const uint2*>(lo);
+        }
+      }
+    }
+  } else {
+    for (int idx = tid; idx < r * W; idx += kThreads) {
+      const int j = idx / W, c = idx % W;
+      if (c0 + c < h) {
+        const float f = slab[j * Wp + c];
+        const int64_t col = c0 + c;
+        Gs[(int64_t)j * h + col] = f;
+        if (out32) out32[((int64_t)s * r + j) * h + col] = f;
+        if (planes) {
+          const __nv_bfloat16 hi = __float2bfloat16_rn(f);
+          planes[(((int64_t)s * 2 + 0) * plane_rows + j) * h + col] = hi;
+          planes[(((int64_t)s * 2 + 1) * plane_rows + j) * h + col] = __float2bfloat16_rn(f - __bfloat162float(hi));
+        }
       }
     }
   }

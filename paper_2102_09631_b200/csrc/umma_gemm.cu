@@ -52,8 +52,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   constexpr int A_BYTES = 128 * 64 * 2;
   constexpr int B_BYTES = B_MN ? (BN / 64) * 8192 : TERMS * BN * 128;
   constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
-  constexpr uint32_t IDESC = instr_desc(128, BN, A_MN, B_MN);
+  // The hi and lo planes of a K-major B operand lie one after the other in a stage, so one MMA of width
+  // TERMS * BN multiplies A by both at once (A is read from shared memory once per k-step); the two halves
+  // of the accumulator are added in the epilogue.
+  constexpr int MMA_N = B_MN ? BN : TERMS * BN;
+  constexpr uint32_t TMEM_COLS = MMA_N < 32 ? 32 : MMA_N;
+  constexpr uint32_t IDESC = instr_desc(128, MMA_N, A_MN, B_MN);
   static_assert(!B_MN || (BN % 64 == 0 && TERMS == 1), "M/N-major B comes in 64-wide chunks, one term");
 
   extern __shared__ uint8_t smem_raw[];
@@ -145,11 +149,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
         for (int k16 = 0; k16 < 4; ++k16) {
           const uint64_t adesc = A_MN ? desc_mn_major(a_addr, k16) : desc_k_major(a_addr, k16);
-#pragma unroll
-          for (int t = 0; t < TERMS; ++t) {
-            const uint64_t bdesc = B_MN ? desc_mn_major(b_addr, k16) : desc_k_major(b_addr + t * BN * 128, k16);
-            umma_bf16(tmem_base, adesc, bdesc, IDESC, (i | k16 | t) != 0 ? 1u : 0u);
-          }
+          const uint64_t bdesc = B_MN ? desc_mn_major(b_addr, k16) : desc_k_major(b_addr, k16);
+          umma_bf16(tmem_base, adesc, bdesc, IDESC, (i | k16) != 0 ? 1u : 0u);
         }
         umma_commit(&empty_bar[stage]);
       }
@@ -172,6 +173,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float v[16];
         if (nkb > 0) {
           tmem_ld16(lane_base + c * 16, v);
+          if constexpr (MMA_N > BN) {  // add the product with the lo plane
+            float w[16];
+            tmem_ld16(lane_base + BN + c * 16, w);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += w[i];
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] = 0.f;
@@ -215,6 +222,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         } else if (nkb > 0) {
           tmem_ld16(lane_base + c * 16, v);
+          if constexpr (MMA_N > BN) {
+            float w[16];
+            tmem_ld16(lane_base + BN + c * 16, w);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += w[i];
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] = 0.f;
@@ -373,7 +386,7 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
   switch (umma_rank_pad(r)) {
     case 16: return launch_umma<16, false, false, 2, EPI_YT, 5>(tmX, tmF, p, grid, "rows_dot_tc", st);
     case 32: return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
-    default: return launch_umma<64, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    default: return launch_umma<64, false, false, 2, EPI_YT, 3>(tmX, tmF, p, grid, "rows_dot_tc", st);
   }
 }
 
@@ -400,7 +413,7 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
   switch (umma_rank_pad(r)) {
     case 16: return launch_umma<16, true, false, 2, EPI_Z, 5>(tmX, tmYt, p, grid, "cols_acc_tc", st);
     case 32: return launch_umma<32, true, false, 2, EPI_Z, 4>(tmX, tmYt, p, grid, "cols_acc_tc", st);
-    default: return launch_umma<64, true, false, 2, EPI_Z, 4>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+    default: return launch_umma<64, true, false, 2, EPI_Z, 3>(tmX, tmYt, p, grid, "cols_acc_tc", st);
   }
 }
 
