@@ -162,6 +162,37 @@ dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* 
                            float* grad, dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Second structured power iteration, at the aggregator (Algorithm 1: after the vertcat, "SPI(Q_i, G_i)" reduces
+ * the stacks of all sites to r rows again, and those r rows are what is broadcast back; Sec. 3.3).  The stacks
+ * take the places of the component matrices -- Pcat^T Qcat is "A^T D" with A = Pcat (K x h_in) and D = Qcat
+ * (K x h_out) -- so this is dad_rank_compress on one slice of K = S*r fp32 rows, with the same arguments, results,
+ * precision (fp64 accumulation) and errors:
+ *     Qhat (r x h_out, orthonormal rows), Phat = (Pcat^T (Qcat Qhat^T))^T (r x h_in), sigma (r, or NULL),
+ * and Phat^T Qhat is the projection of Pcat^T Qcat on the r directions found.  A site then receives
+ * r*(h_in+h_out)*4 bytes (dad_bytes_rank) instead of K*(h_in+h_out)*4.
+ *   Q0  DEVICE, r x h_out fp32 start vectors;  ws >= dad_aggregate_workspace_bytes(h_in, h_out, K, r, iters)
+ */
+size_t dad_aggregate_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, int r, int iters);
+dad_status dad_aggregate_compress(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat,
+                                  int r, int iters, const float* Q0, float* Phat, float* Qhat, float* sigma,
+                                  void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Effective rank (Sec. 3.3.1, last paragraph, and the early stop of Algorithm 2 with theta = 1e-3: components
+ * that carry only noise are not computed or sent, so r is an upper limit on what a site transmits).  The paper's
+ * stop test compares consecutive, mutually orthogonal vectors and cannot trigger as printed; the reading taken
+ * here keeps the leading components of a site while their strength stays above theta times the first one's:
+ *     r_eff[s] = min { j : sigma_s[j] <= theta * sigma_s[0] }   (r if there is no such j; 0 if sigma_s[0] == 0),
+ * the comparison made in fp32 on the fp32 sigma that dad_rank_compress wrote.  Rows j >= r_eff[s] of P_s and Q_s
+ * are set to zero (pass NULL to leave the factors alone), so gather and reconstruct work unchanged and the
+ * dropped components add nothing; the site then transmits dad_bytes_rank(layer, r_eff[s]) bytes.
+ *   sigma DEVICE S x r fp32;  r_eff DEVICE S x int32 (out);  P, Q DEVICE S x r x h_in / h_out fp32 or NULL
+ *   theta in [0, 1].  Only S, h_in, h_out of `layer` are read.
+ */
+dad_status dad_effective_rank(const dad_layer* layer, int r, float theta, const float* sigma, int32_t* r_eff,
+                              float* P, float* Q, void* cuda_stream);
+
+/*
  * Reconstruction without caller scratch (the paper has no counterpart: this is a packaging of
  * dad_reconstruct for hosts that cannot allocate).  Same arguments, results and errors as
  * dad_reconstruct, minus `ws`: the scratch is a fixed array of DAD_STATIC_SCRATCH_BYTES inside the

@@ -297,3 +297,22 @@ void dad_oracle_gather(int S, i64 r, i64 h_in, i64 h_out,
     if (bytes_tx) bytes_tx[s] = dad_oracle_bytes_rank(r, h_in, h_out);
   }
 }
+
+/* ------------------------------------------------------------------------------------
+ * Effective rank of a site's factors (Sec. 3.3.1, last paragraph; the early stop of
+ * Algorithm 2, theta = 1e-3).  As printed the stop test compares consecutive components,
+ * which are orthogonal to each other, and can never fire; the reading taken is: keep the
+ * leading components while sigma_j > theta * sigma_1, drop that one and all later ones.
+ * The decision is an integer taken on fp32 values, so it is made in fp32 here exactly as
+ * the library makes it (fp32 product, fp32 comparison).
+ *   sigma: S x r fp32, r_eff: S (out).
+ * ---------------------------------------------------------------------------------- */
+void dad_oracle_effective_rank(int S, i64 r, const float* sigma, float theta, int32_t* r_eff) {
+  for (int s = 0; s < S; ++s) {
+    const float* sg = sigma + (i64)s * r;
+    const float bar = theta * sg[0];
+    int keep = 0;
+    while (keep < r && sg[keep] > bar) ++keep;
+    r_eff[s] = keep;
+  }
+}

@@ -221,3 +221,45 @@ def rank_dad_layer(A, D, Q0, iters: int):
     Pcat, Qcat, tx = gather(P, Q)
     return {"P": P, "Q": Q, "sigma": sig, "Pcat": Pcat, "Qcat": Qcat, "bytes_tx": tx,
             "grad": reconstruct(Pcat, Qcat)}
+
+
+def aggregate_spi(Pcat, Qcat, Q0, iters: int):
+    """Second structured power iteration at the aggregator (Algorithm 1, "SPI(Q_i, G_i)"): the stacks take
+    the places of the component matrices (A = Pcat, D = Qcat, one slice of K rows).  Returns Phat, Qhat, sigma."""
+    return spi_block(widen(Pcat), widen(Qcat), widen(Q0), iters)
+
+
+def two_stage_layer(A, D, Q0, iters: int, Q0_agg, iters_agg: int):
+    """rank-dAD as Algorithm 1 prints it: per-site SPI, vertcat, SPI of the stacks, Phat^T Qhat."""
+    first = rank_dad_layer(A, D, Q0, iters)
+    Ph, Qh, sg = aggregate_spi(first["Pcat"], first["Qcat"], Q0_agg, iters_agg)
+    r_agg = Ph.shape[0]
+    h_in, h_out = Ph.shape[1], Qh.shape[1]
+    first.update({"Phat": Ph, "Qhat": Qh, "sigma_hat": sg, "grad_hat": reconstruct(Ph, Qh),
+                  "bytes_down": bytes_rank(r_agg, h_in, h_out)})
+    return first
+
+
+def effective_rank(sigma, theta: float) -> np.ndarray:
+    """Leading components kept per site: sigma_j > theta * sigma_1, decided in fp32.  sigma: S x r."""
+    sg = np.ascontiguousarray(np.asarray(sigma, dtype=np.float32))
+    if sg.ndim == 1:
+        sg = sg[None]
+    S, r = sg.shape
+    out = np.zeros(S, dtype=np.int32)
+    L = lib()
+    L.dad_oracle_effective_rank.argtypes = [ctypes.c_int, _i64, ctypes.POINTER(ctypes.c_float), ctypes.c_float,
+                                            ctypes.POINTER(ctypes.c_int32)]
+    L.dad_oracle_effective_rank.restype = None
+    L.dad_oracle_effective_rank(S, r, sg.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), ctypes.c_float(theta),
+                                out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)))
+    return out
+
+
+def truncate(P, Q, r_eff):
+    """Factors with the components j >= r_eff[s] of site s dropped (set to zero)."""
+    P, Q = widen(P).copy(), widen(Q).copy()
+    for s, k in enumerate(np.asarray(r_eff)):
+        P[s, int(k):] = 0.0
+        Q[s, int(k):] = 0.0
+    return P, Q

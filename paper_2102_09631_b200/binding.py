@@ -24,7 +24,7 @@ STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD
 # every symbol include/dad.h declares
 EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
            "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
-           "dad_reconstruct_static",
+           "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
@@ -76,6 +76,13 @@ def lib() -> ctypes.CDLL:
         L.dad_reconstruct.restype = ctypes.c_int
         L.dad_reconstruct_static.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, ctypes.c_int, vp]
         L.dad_reconstruct_static.restype = ctypes.c_int
+        L.dad_aggregate_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int]
+        L.dad_aggregate_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_aggregate_compress.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, ctypes.c_int,
+                                             ctypes.c_int, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.dad_aggregate_compress.restype = ctypes.c_int
+        L.dad_effective_rank.argtypes = [lp, ctypes.c_int, ctypes.c_float, vp, vp, vp, vp, vp]
+        L.dad_effective_rank.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -192,6 +199,25 @@ def dad_reconstruct_static(h_in: int, h_out: int, K: int, Pcat, Qcat, grad, math
     (DAD_STATIC_SCRATCH_BYTES, shared by all calls on the device) stands in for `ws`."""
     st = lib().dad_reconstruct_static(h_in, h_out, K, _ptr(Pcat), _ptr(Qcat), _ptr(grad), math, _stream(stream))
     _check(st, "dad_reconstruct_static")
+
+
+def dad_aggregate_workspace_bytes(h_in: int, h_out: int, K: int, r: int, iters: int) -> int:
+    return int(lib().dad_aggregate_workspace_bytes(h_in, h_out, K, r, iters))
+
+
+def dad_aggregate_compress(h_in: int, h_out: int, K: int, Pcat, Qcat, r: int, iters: int, Q0, Phat, Qhat, sigma, ws,
+                           stream=None):
+    """Second structured power iteration on the stacked factors (the aggregator's SPI of Algorithm 1)."""
+    st = lib().dad_aggregate_compress(h_in, h_out, K, _ptr(Pcat), _ptr(Qcat), r, iters, _ptr(Q0), _ptr(Phat), _ptr(Qhat),
+                                      _ptr(sigma), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_aggregate_compress")
+
+
+def dad_effective_rank(layer: dad_layer, r: int, theta: float, sigma, r_eff, P=None, Q=None, stream=None):
+    """r_eff[s] <- leading components of site s with sigma_j > theta * sigma_1; zeroes the dropped rows of P, Q."""
+    st = lib().dad_effective_rank(ctypes.byref(layer), r, ctypes.c_float(theta), _ptr(sigma), _ptr(r_eff), _ptr(P), _ptr(Q),
+                                  _stream(stream))
+    _check(st, "dad_effective_rank")
 
 
 def dad_check(ws, stream=None):

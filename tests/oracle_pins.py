@@ -369,4 +369,64 @@ def pin_bytes_closed_forms(o):
     assert o.bytes_dad(1 << 20, 1 << 14, 1 << 14, 4) == (1 << 20) * (1 << 15) * 4
 
 
+# --------------------------------------------------------------------------- aggregator SPI, effective rank
+def pin_two_stage_is_spi_of_the_stacks(o):
+    """Algorithm 1 (SPI at the aggregator): Phat^T Qhat is the projection of Pcat^T Qcat = sum_s P_s^T Q_s on
+    r directions; exact once r covers the rank of the stacked product, never better than Eckart-Young, and the
+    optimum in the limit."""
+    rng = _rng(21)
+    S, N, h_in, h_out, r = 3, 9, 10, 8, 2
+    A = rng.standard_normal((S, N, h_in))
+    D = rng.standard_normal((S, N, h_out)) * (1.0 / np.arange(1, h_out + 1))
+    Q0 = rng.standard_normal((S, r, h_out))
+    # aggregator rank 6 = S * r >= rank of the stacked product: nothing is lost
+    out = o.two_stage_layer(A, D, Q0, 2, rng.standard_normal((S * r, h_out)), 1)
+    assert np.linalg.norm(out["grad_hat"] - out["grad"]) <= 1e-10 * np.linalg.norm(out["grad"])
+    # aggregator rank 2 < 6: a rank-2 projection of the stacked product
+    Q0a = rng.standard_normal((2, h_out))
+    target = out["grad"]
+    sv = np.linalg.svd(target, compute_uv=False)
+    last = None
+    for it in (1, 3, 40):
+        o2 = o.two_stage_layer(A, D, Q0, 2, Q0a, it)
+        Ph, Qh = o2["Phat"], o2["Qhat"]
+        assert np.abs(Qh @ Qh.T - np.eye(2)).max() < 1e-12
+        assert np.abs(Ph - (target @ Qh.T).T).max() < 1e-11 * np.abs(target).max() * h_out
+        err2 = np.linalg.norm(target - o2["grad_hat"]) ** 2
+        assert err2 >= np.sum(sv[2:] ** 2) * (1 - 1e-10)
+        if last is not None:
+            assert err2 <= last * (1 + 1e-9)
+        last = err2
+        assert o2["bytes_down"] == 2 * (h_in + h_out) * 4 and list(o2["bytes_tx"]) == [r * (h_in + h_out) * 4] * S
+    assert abs(last - np.sum(sv[2:] ** 2)) < 1e-8 * np.sum(sv ** 2)
+
+
+def pin_effective_rank_worked_cases(o):
+    """Sec. 3.3.1 / Algorithm 2 early stop, theta = 1e-3: hand-worked cases of the rule that is implemented."""
+    with open(os.path.join(GOLDEN, "effective_rank.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            theta, sig, want = [x.strip() for x in line.split("|")]
+            got = o.effective_rank(np.array([float(x) for x in sig.split()], dtype=np.float32), float(theta))
+            assert list(got) == [int(want)], (line, got)
+    # several sites at once are handled independently; truncation zeroes exactly the dropped components
+    sg = np.array([[4, 2, 1e-4, 1], [1, 0.5, 0.25, 0.125]], dtype=np.float32)
+    k = o.effective_rank(sg, 1e-3)
+    assert list(k) == [2, 4]
+    P = np.ones((2, 4, 3))
+    Q = np.ones((2, 4, 5))
+    Pt, Qt = o.truncate(P, Q, k)
+    assert Pt[0, 2:].sum() == 0 and Qt[0, 2:].sum() == 0 and Pt[0, :2].sum() == 6 and Pt[1].sum() == 12
+    # dropping a noise component changes the estimate by no more than its strength
+    rng = _rng(22)
+    A, D, U, V = planted(12, 9, 10, np.array([5.0, 3.0, 1e-5]), seed=23)
+    Pf, Qf, sf = o.spi_block(A, D, rng.standard_normal((3, 10)), 30)
+    keep = o.effective_rank(sf.astype(np.float32), 1e-3)
+    assert list(keep) == [2]
+    Pt, Qt = o.truncate(Pf[None], Qf[None], keep)
+    assert np.linalg.norm(Pt[0].T @ Qt[0] - Pf.T @ Qf) <= 1.0001e-5
+
+
 ALL_PINS = [v for k, v in sorted(globals().items()) if k.startswith("pin_") and callable(v)]

@@ -32,6 +32,8 @@ MUTANTS = [
     ("bytes_dad_ignores_width", "(uint64_t)(h_in + h_out) * (uint64_t)elem_bytes;", "(uint64_t)(h_in + h_out) * 4u;"),
     ("bytes_rank_product", "return (uint64_t)r * (uint64_t)(h_in + h_out) * 4u;", "return (uint64_t)r * (uint64_t)(h_in * h_out) * 4u;"),
     ("bytes_dsgd_sum", "return (uint64_t)h_in * (uint64_t)h_out * 4u;", "return (uint64_t)(h_in + h_out) * 4u;"),
+    ("effective_rank_strict", "while (keep < r && sg[keep] > bar) ++keep;", "while (keep < r && sg[keep] >= bar) ++keep;"),
+    ("effective_rank_vs_previous", "const float bar = theta * sg[0];\n    int keep = 0;\n    while (keep < r && sg[keep] > bar) ++keep;", "int keep = 0;\n    while (keep < r && (keep == 0 ? sg[0] > theta * sg[0] : sg[keep] > theta * sg[keep - 1])) ++keep;"),
     ("gather_reverses_sites", "Pcat[((i64)s * r + j) * h_in + a] = P[((i64)s * r + j) * h_in + a];", "Pcat[((i64)(S - 1 - s) * r + j) * h_in + a] = P[((i64)s * r + j) * h_in + a];"),
 ]
 
