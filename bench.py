@@ -351,31 +351,34 @@ def run_ours(args):
                      "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
                      "layers_per_s": sum(sh.count for sh in cfg.layers) / (ms_total * 1e-3), "per_shape": rows}
 
-    # ---- end to end: inputs start in pinned host memory, the gradient ends there ------------------
+    # ---- end to end: the C-ABI host entry point; inputs start in pinned host memory, the gradient ends there ----
     e2e = None
     if not args.no_e2e:
-        host = [(A.cpu().pin_memory(), D.cpu().pin_memory(), Q0.cpu().pin_memory()) for A, D, Q0 in data[0]]
-        stage = {}
-        for ui, (sh, groups) in enumerate(units):
-            key = (sh.h_in, sh.h_out, groups)
-            if key not in stage:
-                A, D, Q0 = data[0][ui]
-                stage[key] = (torch.empty_like(A), torch.empty_like(D), torch.empty_like(Q0),
-                              torch.empty(groups, sh.h_in, sh.h_out, dtype=torch.float32).pin_memory())
-        h2d = sum(a.numel() * a.element_size() + d.numel() * d.element_size() + q.numel() * 4 for a, d, q in host) * n_super
+        math = B.DAD_F32 if cfg.dtype == "f32" else B.DAD_BF16
+        host, scratch = [], {}
+        for li, sh in enumerate(cfg.layers):      # one pinned input set per layer shape, reused for every such layer
+            seed = wl.seed_for(cfg.index, 900 + li, rank)
+            if cfg.index == 1:
+                A, D = wl.gaussian_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+            else:
+                A, D = wl.decaying_layer(cfg.S, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+            Q0 = wl.start_block(cfg.S, r, sh.h_out, seed, dev)
+            a, d, q = A.cpu().pin_memory(), D.cpu().pin_memory(), Q0.cpu().pin_memory()
+            L1 = B.make_layer(a, d)
+            gh = torch.empty(sh.h_in, sh.h_out, dtype=torch.float32).pin_memory()
+            scratch[li] = torch.empty(B.dad_rank_dad_host_scratch_bytes(L1, r, iters, math), dtype=torch.uint8, device=dev)
+            host.append((L1, a, d, q, gh))
+            del A, D, Q0
+        h2d = sum((a.numel() * a.element_size() + d.numel() * d.element_size() + q.numel() * 4) * sh.count
+                  for (L1, a, d, q, gh), sh in zip(host, cfg.layers)) * cfg.blocks
         d2h = sum(sh.h_in * sh.h_out * 4 for sh in layers) * cfg.blocks
 
         def e2e_step():
-            for b in range(n_super):
-                for ui, (sh, groups) in enumerate(units):
-                    key = (sh.h_in, sh.h_out, groups)
-                    As, Ds, Qs, gh = stage[key]
-                    a, d, q = host[ui]
-                    As.copy_(a, non_blocking=True)
-                    Ds.copy_(d, non_blocking=True)
-                    Qs.copy_(q, non_blocking=True)
-                    plans[key].step(As, Ds, Qs, stream)
-                    gh.copy_(plans[key].grads, non_blocking=True)
+            for b in range(cfg.blocks):
+                for li, sh in enumerate(cfg.layers):
+                    L1, a, d, q, gh = host[li]
+                    for _ in range(sh.count):
+                        B.dad_rank_dad_host(L1, a, d, q, r, iters, math, gh, scratch[li], None, stream)
 
         e2e_step()
         sync_all()
@@ -386,8 +389,9 @@ def run_ours(args):
         e1.record(stream)
         sync_all()
         ems = multi.max_over_ranks(e0.elapsed_time(e1), dev)
-        e2e = {"value": multi.whole_job_rate(n_layers * args.e2e_steps, world, ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+        e2e = {"value": multi.whole_job_rate(n_layers * args.e2e_steps, world, ems * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+               "call": "dad_rank_dad_host per layer (host A, Delta, Q0 in; host gradient out), one stream"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

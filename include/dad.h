@@ -162,6 +162,24 @@ dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* 
                            float* grad, dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The whole per-layer path from HOST memory (Algorithm 1 with the direct sum of outer products at the
+ * aggregator): copies A, D (laid out by `layer`, but in host memory) and Q0 to the device, runs
+ * dad_rank_compress -> dad_gather_factors -> dad_reconstruct there, and copies the h_in x h_out fp32 gradient
+ * back.  Everything is queued on `cuda_stream`; the call does not synchronise and allocates nothing.
+ *   A_host, D_host, Q0_host  HOST (pinned memory for asynchronous copies); strided rows / sites are allowed
+ *   grad_host                HOST, h_in x h_out fp32 (out), valid once the stream has drained
+ *   bytes_tx                 HOST, S entries or NULL: dad_bytes_rank(layer, r) per site
+ *   math                     as for dad_reconstruct
+ *   dev_scratch              DEVICE, 256-byte aligned, >= dad_rank_dad_host_scratch_bytes(layer, r, iters, math):
+ *                            staging for the inputs, the factors, the gradient, and the workspace
+ * Results, precision and errors are those of the three device calls on densely packed copies of the inputs.
+ */
+size_t dad_rank_dad_host_scratch_bytes(const dad_layer* layer, int r, int iters, dad_dtype math);
+dad_status dad_rank_dad_host(const dad_layer* layer, const void* A_host, const void* D_host, const float* Q0_host,
+                             int r, int iters, dad_dtype math, float* grad_host, uint64_t* bytes_tx,
+                             void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+
+/*
  * Second structured power iteration, at the aggregator (Algorithm 1: after the vertcat, "SPI(Q_i, G_i)" reduces
  * the stacks of all sites to r rows again, and those r rows are what is broadcast back; Sec. 3.3).  The stacks
  * take the places of the component matrices -- Pcat^T Qcat is "A^T D" with A = Pcat (K x h_in) and D = Qcat

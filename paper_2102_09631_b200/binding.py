@@ -25,6 +25,7 @@ STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD
 EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
            "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
+           "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host",
            "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
@@ -83,6 +84,11 @@ def lib() -> ctypes.CDLL:
         L.dad_aggregate_compress.restype = ctypes.c_int
         L.dad_effective_rank.argtypes = [lp, ctypes.c_int, ctypes.c_float, vp, vp, vp, vp, vp]
         L.dad_effective_rank.restype = ctypes.c_int
+        L.dad_rank_dad_host_scratch_bytes.argtypes = [lp, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.dad_rank_dad_host_scratch_bytes.restype = ctypes.c_size_t
+        L.dad_rank_dad_host.argtypes = [lp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, u64p, vp,
+                                        ctypes.c_size_t, vp]
+        L.dad_rank_dad_host.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -218,6 +224,22 @@ def dad_effective_rank(layer: dad_layer, r: int, theta: float, sigma, r_eff, P=N
     st = lib().dad_effective_rank(ctypes.byref(layer), r, ctypes.c_float(theta), _ptr(sigma), _ptr(r_eff), _ptr(P), _ptr(Q),
                                   _stream(stream))
     _check(st, "dad_effective_rank")
+
+
+def dad_rank_dad_host_scratch_bytes(layer: dad_layer, r: int, iters: int, math: int) -> int:
+    return int(lib().dad_rank_dad_host_scratch_bytes(ctypes.byref(layer), r, iters, math))
+
+
+def dad_rank_dad_host(layer: dad_layer, A_host, D_host, Q0_host, r: int, iters: int, math: int, grad_host, scratch,
+                      bytes_tx=None, stream=None):
+    """compress -> gather -> reconstruct for HOST tensors (pinned for asynchronous copies); `scratch` is a device
+    uint8 tensor of at least dad_rank_dad_host_scratch_bytes.  Queued on the stream; synchronise before reading."""
+    for t in (A_host, D_host, Q0_host, grad_host):
+        if t.is_cuda:
+            raise ValueError("dad_rank_dad_host takes host tensors")
+    st = lib().dad_rank_dad_host(ctypes.byref(layer), _ptr(A_host), _ptr(D_host), _ptr(Q0_host), r, iters, math,
+                                 _ptr(grad_host), bytes_tx, _ptr(scratch), scratch.numel(), _stream(stream))
+    _check(st, "dad_rank_dad_host")
 
 
 def dad_check(ws, stream=None):

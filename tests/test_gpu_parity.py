@@ -272,3 +272,40 @@ def test_stacked_layers_match_separate_calls(oracle, B):
         ref = oracle.rank_dad_layer(A[sl], D[sl], Q0[sl], iters)
         assert rel(grads[g].double().cpu().numpy(), ref["grad"]) <= TOL[torch.bfloat16]
     assert list(plan.bytes_tx) == [oracle.bytes_rank(r, h_in, h_out)] * (S * groups)
+
+
+def test_host_entry_point_matches_device_path_and_oracle(oracle, B):
+    """dad_rank_dad_host: inputs in (pinned) host memory, gradient back in host memory; same result as the
+    three device calls, bit for bit, for dense and for strided host layouts."""
+    dev = torch.device("cuda:0")
+    S, N, h_in, h_out, r, iters = 3, 260, 128, 192, 8, 2
+    for dtype, tol in ((torch.bfloat16, 2e-2), (torch.float32, 1e-5)):
+        Abig, Dbig = wl.decaying_layer(S, N + 7, h_in + 8, h_out + 16, 55, dtype)
+        Q0 = wl.start_block(S, r, h_out, 55).pin_memory()
+        for strided in (False, True):
+            if strided:
+                A, D = Abig.pin_memory()[:, :N, :h_in], Dbig.pin_memory()[:, :N, :h_out]
+            else:
+                A, D = Abig[:, :N, :h_in].contiguous().pin_memory(), Dbig[:, :N, :h_out].contiguous().pin_memory()
+            L = B.make_layer(A, D)
+            assert (L.ldA == h_in) == (not strided)
+            math = L.dtype
+            scratch = torch.empty(B.dad_rank_dad_host_scratch_bytes(L, r, iters, math), dtype=torch.uint8, device=dev)
+            grad_host = torch.full((h_in, h_out), float("nan")).pin_memory()
+            tx = B.bytes_array(S)
+            B.dad_rank_dad_host(L, A, D, Q0, r, iters, math, grad_host, scratch, tx)
+            torch.cuda.synchronize()
+            Ad, Dd = A.contiguous().to(dev), D.contiguous().to(dev)
+            plan = B.LayerPlan(Ad, Dd, r, iters, zero_copy_gather=True)
+            plan.step(Ad, Dd, Q0.to(dev))
+            B.dad_check(plan.ws)
+            assert torch.equal(plan.grad.cpu(), grad_host)
+            ref = oracle.rank_dad_layer(A.contiguous(), D.contiguous(), Q0, iters)
+            assert rel(grad_host.double().numpy(), ref["grad"]) <= tol
+            assert list(tx) == [int(x) for x in ref["bytes_tx"]]
+    # host-detectable errors come back before anything is queued
+    E = B.STATUS_NAMES.index
+    small = torch.empty(256, dtype=torch.uint8, device=dev)
+    with pytest.raises(B.DadError, match="WORKSPACE"):
+        B.dad_rank_dad_host(L, A, D, Q0, r, iters, math, grad_host, small)
+    assert B.dad_rank_dad_host_scratch_bytes(L, 0, iters, math) == 0
