@@ -61,10 +61,21 @@ __host__ __device__ inline OrthGeom orth_geom(int r, int64_t h, int C) {
   return g;
 }
 
-inline int cluster_size_for(int64_t h) {
-  int C = 1;
-  while (C < 8 && h / (C * 2) >= 128) C *= 2;
-  return C;
+template <int BS>
+inline bool slab_fits(int r, int64_t h, int C) { return orth_geom<BS>(r, h, C).total <= 200 * 1024; }
+
+// CTAs per site.  Every CTA of a cluster repeats the r x r factorisation, so the cluster is kept as small as
+// still fills the GPU with S sites (and as the slab of h / C columns allows); with few sites it grows to 8.
+inline int cluster_size_for(int r, int64_t h, int S) {
+  int best = 0;
+  for (int C = 1; C <= 8; C *= 2) {
+    if (C > 1 && h / C < 128) break;
+    const bool fits = r >= 32 ? slab_fits<8>(r, h, C) : slab_fits<2>(r, h, C);
+    if (!fits) continue;
+    best = C;
+    if ((int64_t)S * C >= 2 * 148) break;
+  }
+  return best;  // 0: no cluster size fits
 }
 }  // namespace
 
@@ -215,12 +226,24 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
       const int i = tid;
       if (i >= j && i < rp) {
         // the diagonal is read from its saved copy: thread j overwrites Lm[j][j] in this very step
-        double d = diag0[j], c = Lm[i * LR + j];
-        for (int l = 0; l < j; ++l) {
-          const double a = Lm[j * LR + l];
-          d -= a * a;
-          c -= Lm[i * LR + l] * a;
+        // four partial sums per dot product: the fp64 dependency chain is a quarter as long
+        double dd[4] = {0.0, 0.0, 0.0, 0.0}, cc[4] = {0.0, 0.0, 0.0, 0.0};
+        int l = 0;
+        for (; l + 4 <= j; l += 4) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const double a = Lm[j * LR + l + u];
+            dd[u] += a * a;
+            cc[u] += Lm[i * LR + l + u] * a;
+          }
         }
+        for (; l < j; ++l) {
+          const double a = Lm[j * LR + l];
+          dd[0] += a * a;
+          cc[0] += Lm[i * LR + l] * a;
+        }
+        const double d = diag0[j] - ((dd[0] + dd[1]) + (dd[2] + dd[3]));
+        const double c = Lm[i * LR + j] - ((cc[0] + cc[1]) + (cc[2] + cc[3]));
         const double orig = diag0[j];
         double piv = d;
         int is_dead = 0, bad = 0;
@@ -368,15 +391,14 @@ static cudaError_t launch_orth_cluster(float* G, int S, int r, int64_t h, int C,
 // Whether the one-launch kernel takes this shape (the slab of a CTA has to fit in shared memory).
 bool orth_cluster_fits(int r, int64_t h) {
   if (h > (int64_t)1 << 30) return false;
-  const int C = cluster_size_for(h);
-  const size_t need = r >= 32 ? orth_geom<8>(r, h, C).total : orth_geom<2>(r, h, C).total;
-  return need <= 200 * 1024;
+  return cluster_size_for(r, h, 1 << 20) > 0;  // the largest admissible cluster decides
 }
 
 // Cholesky-QR (one or two passes, decided on the device) of the rows of G (S x r x h fp32, in place).
 cudaError_t orth_cluster(float* G, int S, int r, int64_t h, double tol, int* status, float* out32,
                          __nv_bfloat16* planes, int plane_rows, cudaStream_t st) {
-  const int C = cluster_size_for(h);
+  const int C = cluster_size_for(r, h, S);
+  if (C == 0) return cudaErrorInvalidValue;
   if (r >= 32)
     return launch_orth_cluster<8>(G, S, r, h, C, tol, status, out32, planes, plane_rows, orth_geom<8>(r, h, C).total, st);
   return launch_orth_cluster<2>(G, S, r, h, C, tol, status, out32, planes, plane_rows, orth_geom<2>(r, h, C).total, st);

@@ -38,7 +38,8 @@ rows_dot_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
     for (int q = 0; q < ROWS; ++q)
 #pragma unroll
       for (int jj = 0; jj < RT; ++jj) acc[q][jj] = TAcc(0);
-    for (int64_t c = lane; c < h; c += 32) {
+#pragma unroll 4
+    for (int64_t c = lane; c < h; c += 32) {  // unrolled: several columns' loads in flight per lane
       TAcc x[ROWS];
 #pragma unroll
       for (int q = 0; q < ROWS; ++q)
@@ -99,6 +100,7 @@ cols_acc_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
     TAcc acc[RT];
 #pragma unroll
     for (int jj = 0; jj < RT; ++jj) acc[jj] = TAcc(0);
+#pragma unroll 4
     for (int64_t n = n0; n < n1; ++n) {
       const TAcc x = (c < h) ? TAcc(to_float(Xs[n * ld + c])) : TAcc(0);
 #pragma unroll
