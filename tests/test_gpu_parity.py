@@ -309,3 +309,28 @@ def test_host_entry_point_matches_device_path_and_oracle(oracle, B):
     with pytest.raises(B.DadError, match="WORKSPACE"):
         B.dad_rank_dad_host(L, A, D, Q0, r, iters, math, grad_host, small)
     assert B.dad_rank_dad_host_scratch_bytes(L, 0, iters, math) == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_degenerate_inputs(oracle, B, dtype):
+    """The degenerate cases of the method: no signal at all (zero errors), identical start vectors (a start
+    block of rank 1), and a single repeated row (a rank-1 gradient compressed with r = 4)."""
+    tol = TOL[dtype]
+    S, N, h_in, h_out, r = 2, 136, 64, 72, 4
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 31, dtype)
+    Q0 = wl.start_block(S, r, h_out, 31)
+    # (a) zero errors: every vector is dropped, factors and gradient are exactly zero
+    g = run_gpu_layer(B, A, torch.zeros_like(D), Q0, r, 2)
+    assert not g["P"].any() and not g["Q"].any() and not g["grad"].any() and not g["full"].any()
+    o = oracle.rank_dad_layer(A, torch.zeros_like(D), Q0, 2)
+    assert not o["grad"].any()
+    # (b) all start vectors equal: the block spans one direction; one vector survives, as in the oracle
+    Q0same = Q0[:, :1].expand(S, r, h_out).contiguous()
+    g, o = check_layer(oracle, B, A, D, Q0same, r, 2, tol, ortho_tol=1e-3)
+    for s in range(S):
+        assert [bool(np.any(g["Q"][s][j] != 0.0)) for j in range(r)] == [True, False, False, False]
+    # (c) every row of the batch the same: A_s^T D_s has rank one, reproduced exactly by the first component
+    A1 = A[:, :1].expand(S, N, h_in).contiguous()
+    D1 = D[:, :1].expand(S, N, h_out).contiguous()
+    g, o = check_layer(oracle, B, A1, D1, Q0, r, 1, tol, ortho_tol=1e-3)
+    assert rel(g["grad"], oracle.full_grad(A1, D1)) <= tol
