@@ -229,11 +229,25 @@ def run_ours(args):
     RB = max(1, min(n_super, args.resident_blocks // G))   # distinct input sets resident in HBM, cycled
     units = [(sh, 1) for sh in layers] if args.no_group else [(sh, sh.count * G) for sh in cfg.layers]
     data = []
+    encoder = None
+    if cfg.index == 3:
+        # config 3 is one real encoder layer: forward/backward with hooks on its six projections (CPU, seeded)
+        proj = wl.encoder_layers(S=cfg.S, seed=wl.seed_for(3, 0, rank))
+        by_shape = {}
+        for name, A, D in proj:
+            by_shape.setdefault((A.shape[2], D.shape[2]), []).append((A, D))
+        encoder = by_shape
     for b in range(RB):
         blk = []
         for ui, (sh, groups) in enumerate(units):
             seed = wl.seed_for(cfg.index, b * len(units) + ui, rank)
-            if cfg.index == 1:
+            if encoder is not None:
+                members = encoder[(sh.h_in, sh.h_out)]
+                pick = [members[(ui + g) % len(members)] for g in range(groups)] if args.no_group else \
+                       [members[g % len(members)] for g in range(groups)]
+                A = torch.cat([m[0] for m in pick]).to(dev)
+                D = torch.cat([m[1] for m in pick]).to(dev)
+            elif cfg.index == 1:
                 A, D = wl.gaussian_layer(cfg.S * groups, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
             else:
                 A, D = wl.decaying_layer(cfg.S * groups, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)

@@ -62,3 +62,32 @@ def gather_counts(local: Sequence[int]) -> List[List[int]]:
     out = [None] * dist.get_world_size()
     dist.all_gather_object(out, list(local))
     return out
+
+
+def allgather_factors(P_local: torch.Tensor, Q_local: torch.Tensor, n_sites: int):
+    """The one exchange step of rank-dAD when the S sites are sharded over ranks (`shard_units`): every rank
+    contributes the factors of its own sites and receives the stacks of all of them, in site order -- the
+    aggregator's vertcat followed by the broadcast, as one all-gather into each rank's own memory.
+
+    P_local: S_local x r x h_in, Q_local: S_local x r x h_out (this rank's sites, in order; S_local may differ
+    by one between ranks).  Returns (Pcat, Qcat) of n_sites*r rows each.  Works on CPU tensors with gloo and on
+    CUDA tensors with nccl; a single process returns its own factors reshaped."""
+    r, h_in, h_out = P_local.shape[1], P_local.shape[2], Q_local.shape[2]
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        assert P_local.shape[0] == n_sites
+        return P_local.reshape(n_sites * r, h_in), Q_local.reshape(n_sites * r, h_out)
+    world, rank = dist.get_world_size(), dist.get_rank()
+    counts = [len(shard_units(n_sites, k, world)) for k in range(world)]
+    assert P_local.shape[0] == counts[rank] == Q_local.shape[0]
+    cap = max(counts)
+    # one buffer per rank holding P then Q, padded to the largest shard so that all contributions have one size
+    mine = torch.zeros(cap * r * (h_in + h_out), dtype=P_local.dtype, device=P_local.device)
+    nP, nQ = counts[rank] * r * h_in, counts[rank] * r * h_out
+    mine[:nP] = P_local.reshape(-1)
+    mine[cap * r * h_in:cap * r * h_in + nQ] = Q_local.reshape(-1)
+    parts = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(parts, mine)
+    Ps = [parts[k][:counts[k] * r * h_in].reshape(counts[k] * r, h_in) for k in range(world)]
+    Qs = [parts[k][cap * r * h_in:cap * r * h_in + counts[k] * r * h_out].reshape(counts[k] * r, h_out)
+          for k in range(world)]
+    return torch.cat(Ps), torch.cat(Qs)

@@ -50,6 +50,42 @@ def test_two_gloo_ranks_agree_on_the_slowest_time(tmp_path):
     assert r0["counts"] == r1["counts"] == [[0, 1, 2, 3], [104, 105, 106]]
 
 
+def _gather_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), LOCAL_RANK=str(rank),
+                      WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import dad_oracle
+    from paper_2102_09631_b200 import multi, workloads as wl
+    multi.init("gloo")
+    S, N, h_in, h_out, r, iters = 5, 12, 10, 9, 2, 2         # 5 sites over 2 ranks: 3 + 2
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 321)
+    Q0 = wl.start_block(S, r, h_out, 321)
+    mine = multi.shard_units(S, rank, world)
+    P, Q, _ = dad_oracle.spi_block(A[mine], D[mine], Q0[mine], iters)      # this rank compresses its own sites
+    Pcat, Qcat = multi.allgather_factors(torch.from_numpy(P), torch.from_numpy(Q), S)
+    grad = dad_oracle.reconstruct(Pcat.numpy(), Qcat.numpy())             # every rank reconstructs the same gradient
+    ref = dad_oracle.rank_dad_layer(A, D, Q0, iters)                       # all sites in one process
+    ok = (np.array_equal(Pcat.numpy(), ref["Pcat"]) and np.array_equal(Qcat.numpy(), ref["Qcat"])
+          and np.array_equal(grad, ref["grad"]))
+    sent = multi.gather_counts([dad_oracle.bytes_rank(r, h_in, h_out)] * len(mine))
+    with open(os.path.join(out_dir, f"g{rank}.json"), "w") as f:
+        json.dump({"ok": bool(ok), "sent": sent, "rows": int(Pcat.shape[0])}, f)
+    multi.barrier()
+    torch.distributed.destroy_process_group()
+
+
+def test_sites_sharded_over_ranks_gather_to_the_same_stacks(tmp_path):
+    """Sites split over two ranks, factors all-gathered: every rank holds exactly the stacks (and hence the
+    gradient) a single process computes; per-site byte counts survive the exchange."""
+    world, port = 2, _free_port()
+    mp.spawn(_gather_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    for rank in range(world):
+        g = json.load(open(tmp_path / f"g{rank}.json"))
+        assert g["ok"] and g["rows"] == 5 * 2
+        assert g["sent"] == [[2 * 19 * 4] * 3, [2 * 19 * 4] * 2]
+
+
 def test_single_rank_helpers_need_no_process_group():
     sys.path.insert(0, ROOT)
     from paper_2102_09631_b200 import multi
