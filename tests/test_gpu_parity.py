@@ -334,3 +334,35 @@ def test_degenerate_inputs(oracle, B, dtype):
     D1 = D[:, :1].expand(S, N, h_out).contiguous()
     g, o = check_layer(oracle, B, A1, D1, Q0, r, 1, tol, ortho_tol=1e-3)
     assert rel(g["grad"], oracle.full_grad(A1, D1)) <= tol
+
+
+def test_layer_step_replays_from_a_cuda_graph(B):
+    """The calls only enqueue work on the caller's stream and keep no host state between calls, so a whole
+    compress -> gather -> reconstruct step can be captured once and replayed on new inputs."""
+    dev = torch.device("cuda:0")
+    S, N, h_in, h_out, r, iters = 4, 512, 256, 384, 16, 2
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 71, torch.bfloat16, dev)
+    A2, D2 = wl.decaying_layer(S, N, h_in, h_out, 72, torch.bfloat16, dev)
+    Q0 = wl.start_block(S, r, h_out, 71, dev)
+    plan = B.LayerPlan(A, D, r, iters)
+    plan.step(A, D, Q0)                       # warm-up outside capture (module load, attribute opt-ins)
+    torch.cuda.synchronize()
+    eager1 = plan.grad.clone()
+    plan.step(A2, D2, Q0)
+    torch.cuda.synchronize()
+    eager2 = plan.grad.clone()
+    Ain, Din = A.clone(), D.clone()            # static input buffers of the graph
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            plan.step(Ain, Din, Q0, stream=side)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(plan.grad, eager1)
+    Ain.copy_(A2)
+    Din.copy_(D2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(plan.grad, eager2)
+    B.dad_check(plan.ws)
