@@ -50,6 +50,8 @@ def parse_args():
                     help="stack the same-shape layers of this many consecutive blocks into one call")
     ap.add_argument("--no-group", action="store_true",
                     help="one call per layer instead of stacking the same-shape layers of a block into one call")
+    ap.add_argument("--cuda-graph", action="store_true",
+                    help="capture one step in a CUDA graph and time its replays (for launch-bound configurations)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -279,6 +281,21 @@ def run_ours(args):
         step()
     for p in plans.values():
         B.dad_check(p.ws)
+    run_step, per_replay = step, None
+    if args.cuda_graph:
+        # launch-bound configurations: capture one whole step once, replay it for every timed step
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        c0 = B.dad_launch_count()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                stream = side
+                step()
+        stream = torch.cuda.current_stream()
+        per_replay = B.dad_launch_count() - c0
+        run_step = graph.replay
+        run_step()
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
     sync_all()
     if rank == 0:
@@ -288,10 +305,10 @@ def run_ours(args):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     for _ in range(args.steps):
-        step()
+        run_step()
     ev1.record(stream)
     sync_all()
-    launches = B.dad_launch_count() - launches0
+    launches = B.dad_launch_count() - launches0 if per_replay is None else per_replay * args.steps
     clocks = sampler.stop() if rank == 0 else None
     ms = multi.max_over_ranks(ev0.elapsed_time(ev1), dev)
     ms_per_step = ms / args.steps
@@ -430,6 +447,7 @@ def run_ours(args):
                            "calls": ("one call per layer" if args.no_group else
                                      f"same-shape layers of {G} consecutive block(s) stacked as extra slices of one call: " +
                                      ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
+                           "launch": "CUDA graph replay" if args.cuda_graph else "stream launches",
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
                 "kernels": kernels, "dad_full_grad": full_grad,
