@@ -135,6 +135,21 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
                              void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The same compression in the form Algorithm 2 prints it, for the regime the paper assumes (batch much smaller
+ * than the layer width, N << h; Sec. 3.3.1): C = A A^T (N x N) is precomputed once per site, every application
+ * of the operator then touches only D and C,  g <- D^T ( C ( D g ) )  (Eq. "reduced_iter" with B = D^T C), and
+ * sigma = sqrt(v^T C v) with v = D g.  A is read twice in all instead of 2*iters + 1 times.  Arguments, results
+ * and errors as dad_rank_compress, with two restrictions: dtype must be DAD_F32 (else DAD_ERR_DTYPE) and
+ * N <= DAD_MAX_GRAM_ROWS (else DAD_ERR_SHAPE).  Products accumulate in fp64.
+ *   ws >= dad_rank_compress_gram_workspace_bytes(layer, r, iters)
+ */
+#define DAD_MAX_GRAM_ROWS 128
+size_t dad_rank_compress_gram_workspace_bytes(const dad_layer* layer, int r, int iters);
+dad_status dad_rank_compress_gram(const dad_layer* layer, const void* A, const void* D, int r, int iters,
+                                  const float* Q0, float* P, float* Q, float* sigma,
+                                  void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Gather at the aggregator (Algorithm 1, the two vertcat lines): site s's factors become rows
  * s*r .. s*r+r-1 of the stacks, and each site is charged what it sent.
  *   P, Q       DEVICE, S x r x h_in and S x r x h_out fp32 (as written by dad_rank_compress)

@@ -316,3 +316,50 @@ void dad_oracle_effective_rank(int S, i64 r, const float* sigma, float theta, in
     r_eff[s] = keep;
   }
 }
+
+/* ------------------------------------------------------------------------------------
+ * Algorithm 2 with its precomputed matrices, for ONE site: C = A A^T (N x N) and
+ * B = D^T C (h_out x N) are formed explicitly, every iteration is G~ = B (D G^T)
+ * (Eq. "reduced_iter") for all r vectors at once, followed by the same orthonormalisation as
+ * spi_block; at the end v_j = D g_j, sigma_j = sqrt(v_j^T C v_j) and P_j = A^T v_j (the
+ * division by sigma is again not made).  This is the form whose cost is O(h N) per vector and
+ * iteration when N << h (Sec. 3.3.1).  Returns 0, or 1 if memory could not be had.
+ * ---------------------------------------------------------------------------------- */
+int dad_oracle_spi_gram_site(i64 N, i64 h_in, i64 h_out, i64 r, int iters,
+                             const double* A, const double* D, const double* Q0,
+                             double* P, double* Q, double* sigma) {
+  double* C = (double*)malloc(sizeof(double) * (size_t)(N * N));
+  double* B = (double*)malloc(sizeof(double) * (size_t)(h_out * N));
+  double* V = (double*)malloc(sizeof(double) * (size_t)(N * r));
+  if (!C || !B || !V) { free(C); free(B); free(V); return 1; }
+  for (i64 n = 0; n < N; ++n)
+    for (i64 m = 0; m < N; ++m) C[n * N + m] = dot(A + n * h_in, A + m * h_in, h_in);
+  for (i64 b = 0; b < h_out; ++b)
+    for (i64 m = 0; m < N; ++m) {
+      double acc = 0.0;
+      for (i64 n = 0; n < N; ++n) acc += D[n * h_out + b] * C[n * N + m];
+      B[b * N + m] = acc;
+    }
+  memcpy(Q, Q0, sizeof(double) * (size_t)(r * h_out));
+  for (int k = 0; k < iters; ++k) {
+    rows_dot(N, h_out, r, D, Q, V);               /* V = D G^T            */
+    for (i64 j = 0; j < r; ++j)                   /* G~_j = B v_j         */
+      for (i64 b = 0; b < h_out; ++b) {
+        double acc = 0.0;
+        for (i64 m = 0; m < N; ++m) acc += B[b * N + m] * V[m * r + j];
+        Q[j * h_out + b] = acc;
+      }
+    dad_oracle_orth(r, h_out, Q, NULL);
+  }
+  rows_dot(N, h_out, r, D, Q, V);
+  cols_acc(N, h_in, r, V, A, P);                  /* P_j = A^T v_j        */
+  if (sigma)
+    for (i64 j = 0; j < r; ++j) {                 /* sigma_j = sqrt(v^T C v) */
+      double acc = 0.0;
+      for (i64 n = 0; n < N; ++n)
+        for (i64 m = 0; m < N; ++m) acc += V[n * r + j] * C[n * N + m] * V[m * r + j];
+      sigma[j] = sqrt(acc > 0.0 ? acc : 0.0);
+    }
+  free(C); free(B); free(V);
+  return 0;
+}

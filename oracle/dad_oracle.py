@@ -263,3 +263,28 @@ def truncate(P, Q, r_eff):
         P[s, int(k):] = 0.0
         Q[s, int(k):] = 0.0
     return P, Q
+
+
+def spi_gram(A, D, Q0, iters: int):
+    """Algorithm 2 with C = A A^T and B = D^T C formed explicitly (the paper's own N << h form), per site.
+    Same arguments and results as spi_block."""
+    single = np.asarray(Q0).ndim == 2 if not hasattr(Q0, "detach") else Q0.dim() == 2
+    A, D = _sites(A, D)
+    Q0 = widen(Q0)
+    if Q0.ndim == 2:
+        Q0 = Q0[None]
+    S, N, h_in = A.shape
+    h_out, r = D.shape[2], Q0.shape[1]
+    P = np.empty((S, r, h_in))
+    Q = np.empty((S, r, h_out))
+    sig = np.empty((S, r))
+    L = lib()
+    L.dad_oracle_spi_gram_site.argtypes = [_i64, _i64, _i64, _i64, ctypes.c_int, _f64p, _f64p, _f64p, _f64p, _f64p, _f64p]
+    L.dad_oracle_spi_gram_site.restype = ctypes.c_int
+    for s in range(S):
+        a, d, q0 = np.ascontiguousarray(A[s]), np.ascontiguousarray(D[s]), np.ascontiguousarray(Q0[s])
+        if L.dad_oracle_spi_gram_site(N, h_in, h_out, r, int(iters), _p(a), _p(d), _p(q0), _p(P[s]), _p(Q[s]), _p(sig[s])):
+            raise MemoryError("dad_oracle_spi_gram_site")
+    if single:
+        return P[0], Q[0], sig[0]
+    return P, Q, sig

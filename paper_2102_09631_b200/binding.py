@@ -25,7 +25,8 @@ STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD
 EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
            "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
-           "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host",
+           "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
+           "dad_rank_compress_gram",
            "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
@@ -89,6 +90,10 @@ def lib() -> ctypes.CDLL:
         L.dad_rank_dad_host.argtypes = [lp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, u64p, vp,
                                         ctypes.c_size_t, vp]
         L.dad_rank_dad_host.restype = ctypes.c_int
+        L.dad_rank_compress_gram_workspace_bytes.argtypes = [lp, ctypes.c_int, ctypes.c_int]
+        L.dad_rank_compress_gram_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_rank_compress_gram.argtypes = [lp, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.dad_rank_compress_gram.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -240,6 +245,20 @@ def dad_rank_dad_host(layer: dad_layer, A_host, D_host, Q0_host, r: int, iters: 
     st = lib().dad_rank_dad_host(ctypes.byref(layer), _ptr(A_host), _ptr(D_host), _ptr(Q0_host), r, iters, math,
                                  _ptr(grad_host), bytes_tx, _ptr(scratch), scratch.numel(), _stream(stream))
     _check(st, "dad_rank_dad_host")
+
+
+DAD_MAX_GRAM_ROWS = 128
+
+
+def dad_rank_compress_gram_workspace_bytes(layer: dad_layer, r: int, iters: int) -> int:
+    return int(lib().dad_rank_compress_gram_workspace_bytes(ctypes.byref(layer), r, iters))
+
+
+def dad_rank_compress_gram(layer: dad_layer, A, D, r: int, iters: int, Q0, P, Q, sigma, ws, stream=None):
+    """dad_rank_compress through C = A A^T (Algorithm 2 as printed; fp32 inputs, N <= DAD_MAX_GRAM_ROWS)."""
+    st = lib().dad_rank_compress_gram(ctypes.byref(layer), _ptr(A), _ptr(D), r, iters, _ptr(Q0), _ptr(P), _ptr(Q),
+                                      _ptr(sigma), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_rank_compress_gram")
 
 
 def dad_check(ws, stream=None):

@@ -429,4 +429,30 @@ def pin_effective_rank_worked_cases(o):
     assert np.linalg.norm(Pt[0].T @ Qt[0] - Pf.T @ Qf) <= 1.0001e-5
 
 
+def pin_spi_gram_form_equals_structured_form(o):
+    """Sec. 3.3.1, Eq. "reduced_iter": iterating B (D g) with B = D^T C, C = A A^T is the same recurrence as
+    gradW^T gradW g, so Algorithm 2 with its precomputed matrices gives the factors of the right-to-left form;
+    and its sigma = sqrt(v^T C v) is the singular value at convergence."""
+    rng = _rng(31)
+    S, N, h_in, h_out, r = 2, 6, 14, 11, 3
+    A = rng.standard_normal((S, N, h_in))
+    D = rng.standard_normal((S, N, h_out))
+    Q0 = rng.standard_normal((S, r, h_out))
+    for iters in (0, 1, 3):
+        Pg, Qg, sg = o.spi_gram(A, D, Q0, iters)
+        Pb, Qb, sb = o.spi_block(A, D, Q0, iters)
+        assert np.abs(Pg - Pb).max() < 1e-9 and np.abs(Qg - Qb).max() < 1e-9 and np.abs(sg - sb).max() < 1e-9
+    # against the explicit operator, one step from one vector
+    gw = A[0].T @ D[0]
+    P1, Q1, s1 = o.spi_gram(A[0], D[0], Q0[0, :1], 1)
+    g = gw.T @ (gw @ Q0[0, 0])
+    g /= np.linalg.norm(g)
+    assert np.abs(Q1[0] - g).max() < 1e-12 and abs(s1[0] - np.linalg.norm(gw @ g)) < 1e-11
+    # converged: sigma are the singular values
+    sig = np.array([6.0, 3.0, 1.0])
+    Ap, Dp, U, V = planted(8, 10, 9, sig, seed=32)
+    Pc, Qc, sc = o.spi_gram(Ap, Dp, rng.standard_normal((3, 9)), 80)
+    assert np.allclose(sc, sig, rtol=1e-9)
+
+
 ALL_PINS = [v for k, v in sorted(globals().items()) if k.startswith("pin_") and callable(v)]

@@ -132,3 +132,55 @@ def test_effective_rank_drops_planted_noise_components(oracle, B):
     ref = oracle.reconstruct(Pt.reshape(S * r, h_in), Qt.reshape(S * r, h_out))
     assert rel(plan.grads[0].double().cpu().numpy(), ref) <= 1e-5
     assert sum(B.dad_bytes_rank(L, int(k)) for k in keep.cpu()) * 2 == S * B.dad_bytes_rank(L, r)
+
+
+@pytest.mark.parametrize("S,N,h_in,h_out,r,iters", [
+    (2, 16, 64, 32, 4, 2),        # config 1
+    (4, 64, 784, 1024, 8, 3),     # the paper's own setting: batch 64 per site, 784-1024-1024-10 MLP
+    (4, 128, 1024, 1024, 8, 3),   # config-2 middle layer, N = 128 = the largest batch this form takes
+    (3, 37, 200, 10, 8, 2),       # narrow output (r close to h_out), odd sizes
+    (2, 5, 48, 40, 8, 1),         # batch smaller than r: exact, surplus vectors zero
+])
+def test_gram_form_matches_oracle_and_structured_form(oracle, B, S, N, h_in, h_out, r, iters):
+    """dad_rank_compress_gram (C = A A^T precomputed, Algorithm 2 as printed) against the oracle's literal
+    Algorithm 2 and against dad_rank_compress on the same inputs."""
+    dev = torch.device("cuda:0")
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 400 + N, torch.float32)
+    Q0 = wl.start_block(S, r, h_out, 400 + N)
+    Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
+    L = B.make_layer(Ad, Dd)
+    P, Q, sg = (torch.empty(S, r, h_in, device=dev), torch.empty(S, r, h_out, device=dev), torch.empty(S, r, device=dev))
+    ws = B.new_workspace(B.dad_rank_compress_gram_workspace_bytes(L, r, iters), dev)
+    B.dad_rank_compress_gram(L, Ad, Dd, r, iters, Q0d, P, Q, sg, ws)
+    B.dad_check(ws)
+    Po, Qo, so = oracle.spi_gram(A, D, Q0, iters)
+    P2, Q2, s2 = (torch.empty_like(P), torch.empty_like(Q), torch.empty_like(sg))
+    ws2 = B.new_workspace(B.dad_workspace_bytes(L, r, iters), dev)
+    B.dad_rank_compress(L, Ad, Dd, r, iters, Q0d, P2, Q2, s2, ws2)
+    B.dad_check(ws2)
+    Pn, Qn = P.double().cpu().numpy(), Q.double().cpu().numpy()
+    for s in range(S):
+        ref = Po[s].T @ Qo[s]
+        assert rel(Pn[s].T @ Qn[s], ref) <= 1e-5
+        assert rel(P2[s].double().cpu().numpy().T @ Q2[s].double().cpu().numpy(), ref) <= 1e-5
+        live = [j for j in range(r) if np.any(Qo[s][j] != 0.0)]
+        assert [j for j in range(r) if np.any(Qn[s][j] != 0.0)] == live
+        assert np.linalg.norm(Qn[s][live] @ Qn[s][live].T - np.eye(len(live))) <= 1e-4
+        scale = max(so[s].max(), 1e-300)
+        assert np.abs(sg[s].cpu().numpy() - so[s]).max() <= 1e-5 * scale     # sqrt(v^T C v)
+        assert np.abs(s2[s].cpu().numpy() - so[s]).max() <= 1e-5 * scale     # ||P_j||: the same number
+
+
+def test_gram_form_refuses_what_it_does_not_take(B):
+    dev = torch.device("cuda:0")
+    A = torch.zeros(1, 129, 16, device=dev)
+    D = torch.zeros(1, 129, 16, device=dev)
+    L = B.make_layer(A, D)
+    assert B.dad_rank_compress_gram_workspace_bytes(L, 4, 1) == 0
+    buf = torch.empty(4, 16, device=dev)
+    ws = B.new_workspace(1 << 20, dev)
+    with pytest.raises(B.DadError, match="SHAPE"):
+        B.dad_rank_compress_gram(L, A, D, 4, 1, buf, buf, buf, None, ws)
+    Lb = B.make_layer(A[:, :64].bfloat16(), D[:, :64].bfloat16())
+    with pytest.raises(B.DadError, match="DTYPE"):
+        B.dad_rank_compress_gram(Lb, A, D, 4, 1, buf, buf, buf, None, ws)

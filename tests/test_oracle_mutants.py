@@ -32,6 +32,9 @@ MUTANTS = [
     ("bytes_dad_ignores_width", "(uint64_t)(h_in + h_out) * (uint64_t)elem_bytes;", "(uint64_t)(h_in + h_out) * 4u;"),
     ("bytes_rank_product", "return (uint64_t)r * (uint64_t)(h_in + h_out) * 4u;", "return (uint64_t)r * (uint64_t)(h_in * h_out) * 4u;"),
     ("bytes_dsgd_sum", "return (uint64_t)h_in * (uint64_t)h_out * 4u;", "return (uint64_t)(h_in + h_out) * 4u;"),
+    ("gram_form_C_not_symmetric_use", "for (i64 n = 0; n < N; ++n) acc += D[n * h_out + b] * C[n * N + m];", "for (i64 n = 0; n < N; ++n) acc += D[n * h_out + b] * C[n * N + (m + 1) % N];"),
+    ("gram_form_sigma_without_C", "acc += V[n * r + j] * C[n * N + m] * V[m * r + j];", "acc += (n == m) ? V[n * r + j] * V[m * r + j] : 0.0;"),
+    ("gram_form_skips_orth", "        Q[j * h_out + b] = acc;\n      }\n    dad_oracle_orth(r, h_out, Q, NULL);", "        Q[j * h_out + b] = acc;\n      }\n    ;"),
     ("effective_rank_strict", "while (keep < r && sg[keep] > bar) ++keep;", "while (keep < r && sg[keep] >= bar) ++keep;"),
     ("effective_rank_vs_previous", "const float bar = theta * sg[0];\n    int keep = 0;\n    while (keep < r && sg[keep] > bar) ++keep;", "int keep = 0;\n    while (keep < r && (keep == 0 ? sg[0] > theta * sg[0] : sg[keep] > theta * sg[keep - 1])) ++keep;"),
     ("gather_reverses_sites", "Pcat[((i64)s * r + j) * h_in + a] = P[((i64)s * r + j) * h_in + a];", "Pcat[((i64)(S - 1 - s) * r + j) * h_in + a] = P[((i64)s * r + j) * h_in + a];"),
