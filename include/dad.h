@@ -167,8 +167,12 @@ dad_status dad_gather_factors(const dad_layer* layer, int r, const float* P, con
  *     grad[a][b] = sum_k Pcat[k][a] * Qcat[k][b].
  *   Pcat, Qcat DEVICE, K x h_in and K x h_out fp32, contiguous, 16-byte aligned
  *   grad       DEVICE, h_in x h_out fp32 (out)
- *   math       DAD_F32: fp32 FMA.  DAD_BF16: tensor cores, factors rounded to bf16, fp32
- *              accumulation (for layers whose inputs were bf16 already).
+ *   math       DAD_F32: fp32 FMA.  DAD_BF16: tensor cores with fp32 accumulation; each fp32
+ *              factor enters as a two-term bf16 split x = hi + lo and the product is
+ *              hi*hi + hi*lo + lo*hi (one contraction of length 3K), so the result carries about
+ *              16 significant bits of the factors (the dropped lo*lo term is 2^-16 relative).
+ *              Needs h_in and h_out multiples of 8; otherwise DAD_BF16 falls back to the
+ *              fp32 FMA kernel (still on the device).
  *   ws         DEVICE scratch of ws_bytes >= dad_reconstruct_workspace_bytes(h_in, h_out, K),
  *              may be NULL when that is 0
  */

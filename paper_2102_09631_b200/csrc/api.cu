@@ -354,13 +354,13 @@ dad_status dad_gather_factors(const dad_layer* L, int r, const float* P, const f
 }
 
 static bool reconstruct_tc(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
-  return math == DAD_BF16 && h_in % 8 == 0 && h_out % 8 == 0 && K <= 0x7fffffff && tmap_encoder_available();
+  return math == DAD_BF16 && h_in % 8 == 0 && h_out % 8 == 0 && 3 * K <= 0x7fffffff && tmap_encoder_available();
 }
 
 size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
   if (h_in < 1 || h_out < 1 || K < 1) return 0;
   if (!reconstruct_tc(h_in, h_out, K, math)) return 0;
-  return gemm_ws_layout(h_in, h_out, 1, K, true).total;
+  return gemm_ws_layout(h_in, h_out, 1, 3 * K, true).total;
 }
 
 dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat, float* grad,
@@ -372,15 +372,15 @@ dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* 
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
   if (reconstruct_tc(h_in, h_out, K, math)) {
-    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, K, true);
+    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, 3 * K, true);  // three bf16 products, one contraction
     if (!ws) return DAD_ERR_NULL;
     if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
     if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
     __nv_bfloat16* Xb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Xb);
     __nv_bfloat16* Yb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Yb);
-    err = f32_to_bf16(Pcat, Xb, (size_t)K * h_in, st);
-    if (err == cudaSuccess) err = f32_to_bf16(Qcat, Yb, (size_t)K * h_out, st);
-    if (err == cudaSuccess) err = run_gemm_tc(Xb, h_in, K * h_in, Yb, h_out, K * h_out, 1, K, h_in, h_out, grad, (char*)ws, w, st);
+    err = stack_split3(Pcat, (size_t)K * h_in, Xb, Qcat, (size_t)K * h_out, Yb, st);
+    if (err == cudaSuccess)
+      err = run_gemm_tc(Xb, h_in, 3 * K * h_in, Yb, h_out, 3 * K * h_out, 1, 3 * K, h_in, h_out, grad, (char*)ws, w, st);
   } else {
     err = gemm_tn_simt(DAD_F32, Pcat, h_in, 0, Qcat, h_out, 0, 1, K, h_in, h_out, grad, st);
   }

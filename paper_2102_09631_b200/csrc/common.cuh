@@ -120,7 +120,8 @@ cudaError_t row_norms(const T* M, int64_t rows, int64_t h, float* out, cudaStrea
 // planes[s][0/1][j][c] = hi / lo bf16 terms of in[s][j][c]  (j < r; plane_rows >= r rows per plane)
 cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16* planes, int plane_rows,
                          cudaStream_t st);
-cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStream_t st);
+cudaError_t stack_split3(const float* P, size_t nP, __nv_bfloat16* X3, const float* Q, size_t nQ, __nv_bfloat16* Y3,
+                         cudaStream_t st);
 
 // ---- tensor-core launchers (umma_gemm.cu) -------------------------------------------------------
 bool tmap_encoder_available();

@@ -218,7 +218,8 @@ def test_reconstruct_and_full_grad_at_full_size_on_sampled_rows(oracle, B):
         ws = B.new_workspace(B.dad_reconstruct_workspace_bytes(h_in, h_out, K, math), dev)
         B.dad_reconstruct(h_in, h_out, K, Pcat.to(dev), Qcat.to(dev), grad, math, ws)
         ref = oracle.reconstruct(Pcat[:, rows], Qcat)
-        assert rel(grad[rows].double().cpu().numpy(), ref) <= (1e-5 if math == B.DAD_F32 else 2e-2)
+        # tensor-core reconstruction multiplies two-term bf16 splits (three products): ~2^-16 relative
+        assert rel(grad[rows].double().cpu().numpy(), ref) <= (1e-5 if math == B.DAD_F32 else 1e-4)
     S, N = 16, 4096
     A, D = wl.decaying_layer(S, N, h_in, h_out, 32, torch.bfloat16, device=dev)
     L = B.make_layer(A, D)
