@@ -97,14 +97,13 @@ GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_ope
   size_t off = 0;
   w.status = off;
   off += 256;
-  const int bn = umma_gemm_bn(hy);
-  const size_t tiles = (size_t)(ceil_div(hx, 128) * ceil_div(hy, bn));
-  const int splits = umma_gemm_splits(hx, hy, ceil_div(N, 64) * S);
+  const GemmPlan g = umma_gemm_plan(hx, hy, S, N);
+  const size_t tiles = (size_t)g.tiles;
   w.n_counters = tiles;
   w.counters = off;
   off = align_up(off + tiles * sizeof(unsigned), 256);
   w.partial = off;
-  off = align_up(off + (splits > 1 ? tiles * (size_t)splits * 128 * (size_t)bn * 4 : 0), 256);
+  off = align_up(off + (g.splits > 1 ? tiles * (size_t)g.splits * (size_t)g.bm * (size_t)g.bn * 4 : 0), 256);
   w.Xb = w.Yb = off;
   if (convert_operands) {
     w.Xb = off;
@@ -243,10 +242,11 @@ static cudaError_t run_gemm_tc(const void* X, int64_t ldX, int64_t strideX, cons
   cudaError_t err = cudaMemsetAsync(ws + w.status + 4, 0, w.counters + w.n_counters * sizeof(unsigned) - w.status - 4, st);
   if (err != cudaSuccess) return err;
   CUtensorMap tmX, tmY;
-  if (!make_tmap_bf16_3d(&tmX, X, hx, N, S, (uint64_t)ldX * 2, (uint64_t)strideX * 2, 64, 64) ||
-      !make_tmap_bf16_3d(&tmY, Y, hy, N, S, (uint64_t)ldY * 2, (uint64_t)strideY * 2, 64, 64))
+  const GemmPlan g = umma_gemm_plan(hx, hy, S, N);
+  if (!make_tmap_bf16_3d(&tmX, X, hx, N, S, (uint64_t)ldX * 2, (uint64_t)strideX * 2, 64, (uint32_t)g.bk) ||
+      !make_tmap_bf16_3d(&tmY, Y, hy, N, S, (uint64_t)ldY * 2, (uint64_t)strideY * 2, 64, (uint32_t)g.bk))
     return cudaErrorInvalidValue;
-  return umma_gemm_tn(tmX, tmY, S, N, hx, hy, C, reinterpret_cast<float*>(ws + w.partial),
+  return umma_gemm_tn(tmX, tmY, g, hx, hy, C, reinterpret_cast<float*>(ws + w.partial),
                       reinterpret_cast<unsigned*>(ws + w.counters), reinterpret_cast<int*>(ws + w.status + 4), st);
 }
 

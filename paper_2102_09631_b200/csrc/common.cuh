@@ -129,14 +129,19 @@ bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t
                        uint64_t s2_bytes, uint32_t box0, uint32_t box1);
 int umma_rank_pad(int r);
 int umma_cols_acc_splits(int S, int64_t N, int64_t h);
-int umma_gemm_bn(int64_t hy);
-int umma_gemm_splits(int64_t hx, int64_t hy, int64_t k_blocks);
+// Geometry of the dense product C = X^T Y (hx x hy, contraction over S sites of N rows): tile bm x bn, stages of
+// bk contraction rows (the row count of the operands' TMA boxes), `splits` CTAs share a tile's contraction.
+struct GemmPlan {
+  int bm, bn, bk, splits;
+  int64_t tiles, k_blocks, kb_per_site;
+};
+GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N);
 cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S, int64_t N, int64_t h, int r,
                           __nv_bfloat16* yt_planes, int64_t ld_planes, int* status, cudaStream_t st);
 cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,
                           float* out2, __nv_bfloat16* planes, int64_t ld_planes, float* partial, unsigned* counters,
                           int* status, cudaStream_t st);
-cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, int S, int64_t N, int64_t hx, int64_t hy,
+cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& plan, int64_t hx, int64_t hy,
                          float* C, float* partial, unsigned* counters, int* status, cudaStream_t st);
 
 }  // namespace dad

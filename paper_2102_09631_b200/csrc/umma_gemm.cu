@@ -28,6 +28,12 @@ using namespace sm100;
 
 enum : int { EPI_YT = 0, EPI_Z = 1, EPI_C = 2 };
 
+// 256 x 256 dense-product kernel: contraction rows per stage, stages (3 x 64 KB of shared memory), and the
+// shortest contraction it is used for (below that the output write dominates and 128-row tiles fill more SMs).
+constexpr int kGemm256BK = 64;
+constexpr int kGemm256Stages = 3;
+constexpr int kGemm256MinRows = 4096;
+
 struct UmmaParams {
   int m_extent;      // valid rows of D: N (rows_dot), h (cols_acc), h_in (gemm_tn)
   int n_extent;      // valid columns of D: r, or h_out
@@ -292,6 +298,189 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
+// Dense product C = X^T Y for long contractions (the dAD gradient, K = S*N): one CTA owns a 256 x 256
+// tile as two 128 x 256 accumulators that fill tensor memory (512 columns).  Both MMAs of a k-step read
+// the same B operand, so a CTA fetches 64 KB per 64-deep block for 2 * 256 * 256 * 64 flops: two thirds of
+// the bytes per flop of the 128 x 256 tile, and the same bytes in flight cover a 1.5x longer stretch of
+// MMA time.  Stages are BK contraction rows deep (BK = 32: more, finer stages in the same shared memory).
+// Same roles, bounded waits, split reduction and teardown as umma_kernel.
+template <int BK, int STAGES>
+__global__ void __launch_bounds__(192)
+umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const UmmaParams p) {
+  constexpr int CHUNK = BK * 128;          // [BK k-rows][64 bf16 along M or N]
+  constexpr int A_BYTES = 4 * CHUNK;       // 256 rows of the tile
+  constexpr int STAGE_BYTES = 8 * CHUNK;   // A and B
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t IDESC = instr_desc(128, 256, true, true);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag, issued_s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tile = blockIdx.x;
+  const int n_tile = blockIdx.y / p.splits, split = blockIdx.y % p.splits;
+  const int m0 = m_tile * 256, n0 = n_tile * 256;
+  const int kb0 = split * p.kb_per_split;
+  const int kb1 = (kb0 + p.kb_per_split < p.k_blocks) ? kb0 + p.kb_per_split : p.k_blocks;
+  const int nkb = kb1 > kb0 ? kb1 - kb0 : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&accum_bar, 1);
+    abort_flag = 0;
+    issued_s = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_s, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  volatile int* abortp = &abort_flag;
+
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmA);
+      prefetch_tmap(&tmB);
+      for (int i = 0; i < nkb; ++i) {
+        const int stage = i % STAGES;
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp)) break;
+        mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+        uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
+        uint8_t* b_dst = a_dst + A_BYTES;
+        const int kb = kb0 + i;
+        const int bz = kb / p.kb_per_site;
+        const int kcoord = (kb % p.kb_per_site) * BK;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tma_load_3d(a_dst + c * CHUNK, &tmA, &full_bar[stage], m0 + c * 64, kcoord, bz);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tma_load_3d(b_dst + c * CHUNK, &tmB, &full_bar[stage], n0 + c * 64, kcoord, bz);
+        issued_s = i + 1;
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      for (int i = 0; i < nkb; ++i) {
+        const int stage = i % STAGES;
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        if (!mbar_wait(&full_bar[stage], ph, abortp)) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+        const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+        for (int k16 = 0; k16 < BK / 16; ++k16) {
+          const uint64_t bdesc = smem_desc(b_addr + (uint32_t)k16 * 2048u, CHUNK, 1024u);
+          const uint32_t acc = (i | k16) != 0 ? 1u : 0u;
+          umma_bf16(tmem_base, smem_desc(a_addr + (uint32_t)k16 * 2048u, CHUNK, 1024u), bdesc, IDESC, acc);
+          umma_bf16(tmem_base + 256u, smem_desc(a_addr + 2u * CHUNK + (uint32_t)k16 * 2048u, CHUNK, 1024u), bdesc, IDESC, acc);
+        }
+        umma_commit(&empty_bar[stage]);
+      }
+      umma_commit(&accum_bar);
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;  // row inside each 128-row half
+    const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+    const bool ok = mbar_wait(&accum_bar, 0u, abortp);
+    tc_fence_after();
+    const int tiles_n = gridDim.y / p.splits;
+    const int64_t tile_lin = (int64_t)m_tile * tiles_n + n_tile;
+    // With a split contraction every CTA stores its partial tile and gemm256_reduce sums them in split
+    // order; otherwise the tile goes straight to C.
+    float* my_partial = p.splits > 1 ? p.partial + (tile_lin * p.splits + split) * (int64_t)(256 * 256) : nullptr;
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < 32; ++c) {  // chunk c: half c / 16 of the tile, columns (c % 16) * 16 .. +15
+        const int half = c / 16, col = (c % 16) * 16;
+        float v[16];
+        if (nkb > 0) {
+          tmem_ld16(lane_base + (uint32_t)c * 16u, v);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
+        if (my_partial) {
+          float4* dst = reinterpret_cast<float4*>(my_partial + (half * 128 + row) * 256 + col);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        } else {
+          const int64_t gm = (int64_t)m0 + half * 128 + row;
+          if (gm < p.m_extent) {
+            float* dst = p.out_f32 + gm * p.ld_out + n0 + col;
+            if (n0 + col + 16 <= p.n_extent && (p.ld_out & 3) == 0) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                if (n0 + col + i < p.n_extent) dst[i] = v[i];
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    if (threadIdx.x == 0) {
+      const int issued = issued_s;
+      const int first = issued > STAGES ? issued - STAGES : 0;
+      for (int i = first; i < issued; ++i) {
+        uint64_t* bar = &full_bar[i % STAGES];
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(bar, ph); ++t) {
+        }
+      }
+      if (p.status) *p.status = (int)DAD_ERR_TIMEOUT;
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// C[m][n] = sum over splits, in split order, of the partial tiles umma_gemm256_kernel stored
+// ([tile][split][256][256] fp32): four columns per thread, the whole GPU instead of one CTA per tile.
+__global__ void __launch_bounds__(256)
+gemm256_reduce_kernel(const float* __restrict__ partial, int splits, int m_extent, int n_extent, float* __restrict__ C) {
+  const int n4 = n_extent / 4;  // n_extent is a multiple of 8 on this path
+  const int tiles_n = (n_extent + 255) / 256;
+  const int64_t total = (int64_t)m_extent * n4;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int m = (int)(idx / n4), n = (int)(idx % n4) * 4;
+    const int64_t tile = (int64_t)(m / 256) * tiles_n + n / 256;
+    const float* src = partial + tile * splits * (int64_t)(256 * 256) + (m % 256) * 256 + n % 256;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < splits; ++s) {
+      const float4 t = __ldcg(reinterpret_cast<const float4*>(src + (int64_t)s * (256 * 256)));
+      acc.x += t.x;
+      acc.y += t.y;
+      acc.z += t.z;
+      acc.w += t.w;
+    }
+    *reinterpret_cast<float4*>(C + (int64_t)m * n_extent + n) = acc;
+  }
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -417,38 +606,89 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
   }
 }
 
-// Tile width of the dense product: 256 columns keep the MMAs under the shared-memory read rate
-// (a 128 x 128 x 16 MMA needs 128 B/clk of operands, a 128 x 256 x 16 one 96 B/clk).
-int umma_gemm_bn(int64_t hy) { return hy > 128 ? 256 : 128; }
-
-int umma_gemm_splits(int64_t hx, int64_t hy, int64_t k_blocks) {
-  const int64_t tiles = ceil_div(hx, 128) * ceil_div(hy, umma_gemm_bn(hy));
-  int64_t splits = 148 / tiles;
-  if (splits > k_blocks / 8) splits = k_blocks / 8;
+// Geometry of the dense product.  Long contractions (the dAD gradient) over outputs at least 256 x 256 take
+// the 256 x 256 two-accumulator kernel; everything else 128 x BN tiles, BN = 256 where the output is wide
+// enough (a 128 x 128 x 16 MMA needs 128 B/clk of operands from shared memory, a 128 x 256 x 16 one
+// 96 B/clk).  Splits of the contraction fill the 148 SMs when the tiles alone do not.
+GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N) {
+  GemmPlan g;
+  const bool big = hx >= 256 && hy >= 256 && N * S >= kGemm256MinRows;
+  int64_t min_blocks;
+  if (big) {
+    g.bm = 256;
+    g.bn = 256;
+    g.bk = kGemm256BK;
+    g.tiles = ceil_div(hx, 256) * ceil_div(hy, 256);
+    min_blocks = 512 / g.bk;
+  } else {
+    g.bm = 128;
+    g.bn = hy > 128 ? 256 : 128;
+    g.bk = 64;
+    g.tiles = ceil_div(hx, 128) * ceil_div(hy, g.bn);
+    min_blocks = 8;
+  }
+  g.kb_per_site = ceil_div(N, g.bk);
+  g.k_blocks = g.kb_per_site * S;
+  int64_t splits = 148 / g.tiles;
+  if (splits > g.k_blocks / min_blocks) splits = g.k_blocks / min_blocks;
   if (splits > 32) splits = 32;
   if (splits < 1) splits = 1;
-  const int64_t per = ceil_div(k_blocks, splits);
-  return (int)ceil_div(k_blocks, per);
+  const int64_t per = ceil_div(g.k_blocks, splits);
+  g.splits = (int)ceil_div(g.k_blocks, per);  // no empty split
+  return g;
 }
 
-// C (hx x hy, fp32) <- sum over sites and rows of X^T Y.  tmX: (hx, N, S) box 64 x 64; tmY: (hy, N, S) box 64 x 64.
-cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, int S, int64_t N, int64_t hx, int64_t hy,
+template <int BK, int STAGES>
+static cudaError_t launch_gemm256(const CUtensorMap& tmA, const CUtensorMap& tmB, const UmmaParams& p, dim3 grid,
+                                  cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * 8 * BK * 128 + 1024;
+  auto kernel = umma_gemm256_kernel<BK, STAGES>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(192, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const bool timed = g_timing.load(std::memory_order_relaxed);
+  if (timed) timing_mark("gemm_tn_tc", st, true);
+  err = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+  if (timed) timing_mark("gemm_tn_tc", st, false);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return err;
+}
+
+// C (hx x hy, fp32) <- sum over sites and rows of X^T Y.  tmX: (hx, N, S), tmY: (hy, N, S), boxes 64 x plan.bk.
+cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& g, int64_t hx, int64_t hy,
                          float* C, float* partial, unsigned* counters, int* status, cudaStream_t st) {
   UmmaParams p{};
   p.m_extent = (int)hx;
   p.n_extent = (int)hy;
-  p.kb_per_site = (int)ceil_div(N, 64);
-  p.k_blocks = p.kb_per_site * S;
-  p.splits = umma_gemm_splits(hx, hy, p.k_blocks);
-  p.kb_per_split = (int)ceil_div(p.k_blocks, p.splits);
+  p.kb_per_site = (int)g.kb_per_site;
+  p.k_blocks = (int)g.k_blocks;
+  p.splits = g.splits;
+  p.kb_per_split = (int)ceil_div(g.k_blocks, g.splits);
   p.out_f32 = C;
   p.ld_out = hy;
   p.partial = partial;
   p.counters = counters;
   p.status = status;
-  const int bn = umma_gemm_bn(hy);
-  dim3 grid((unsigned)ceil_div(hx, 128), (unsigned)(ceil_div(hy, bn) * p.splits), 1);
-  if (bn == 256) return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+  dim3 grid((unsigned)ceil_div(hx, g.bm), (unsigned)(ceil_div(hy, g.bn) * g.splits), 1);
+  if (g.bm == 256) {
+    cudaError_t err = launch_gemm256<kGemm256BK, kGemm256Stages>(tmX, tmY, p, grid, st);
+    if (err != cudaSuccess || g.splits == 1) return err;
+    const int64_t quads = hx * hy / 4;
+    unsigned blocks = (unsigned)(quads / 256 < 148 * 8 ? ceil_div(quads, 256) : 148 * 8);
+    DAD_LAUNCH(err, "gemm_tn_reduce", gemm256_reduce_kernel, blocks, 256, 0, st, (const float*)partial, g.splits, (int)hx,
+               (int)hy, C);
+    return err;
+  }
+  if (g.bn == 256) return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st);
   return launch_umma<128, true, true, 1, EPI_C, 6>(tmX, tmY, p, grid, "gemm_tn_tc", st);
 }
 

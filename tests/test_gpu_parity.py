@@ -131,6 +131,29 @@ def test_shape_slices(oracle, B, N, h_in, h_out, r, iters, dtype):
     check_layer(oracle, B, A, D, Q0, r, iters, TOL[dtype], ortho_tol=1e-3 if dtype == torch.bfloat16 else 1e-4)
 
 
+@pytest.mark.parametrize("S,N,h_in,h_out", [
+    (5, 1000, 520, 776),    # ragged 256 x 256 tiles, rows per site no multiple of a 64-row stage, split contraction
+    (3, 1400, 256, 264),    # one full tile and a sliver
+    (9, 512, 1024, 256),    # whole tiles, one stage-aligned site after the other
+])
+def test_full_grad_long_contraction(oracle, B, S, N, h_in, h_out):
+    """The dAD gradient sum_s A_s^T D_s (Section 3.2) on the tensor cores where the contraction is long
+    (S*N >= 4096 rows): bf16 products are exact in fp32, so only the fp32 accumulation order separates the
+    result from the fp64 oracle -- a far tighter bar than the 2e-2 of the bf16 path as a whole."""
+    dev = torch.device("cuda:0")
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 77 + N, torch.bfloat16)
+    L = B.make_layer(A.to(dev), D.to(dev))
+    ws = B.new_workspace(B.dad_workspace_bytes(L, 1, 0), dev)
+    grads = []
+    for _ in range(2):
+        grad = torch.full((h_in, h_out), float("nan"), device=dev)
+        B.dad_full_grad(L, A.to(dev), D.to(dev), grad, None, ws)
+        B.dad_check(ws)
+        grads.append(grad.cpu())
+    assert torch.equal(grads[0], grads[1])  # ordered split reduction: bit-identical runs
+    assert rel(grads[0].double().numpy(), oracle.full_grad(A, D)) <= 1e-4
+
+
 def test_factors_match_on_separated_spectrum(oracle, B):
     """With well separated singular values and enough iterations each vector is determined up to
     rounding (thin QR with positive diagonal fixes the sign), so the raw factors agree too."""
