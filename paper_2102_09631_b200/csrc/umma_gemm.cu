@@ -622,7 +622,7 @@ GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N) {
     min_blocks = 512 / g.bk;
   } else {
     g.bm = 128;
-    g.bn = hy > 128 ? 256 : 128;
+    g.bn = (hy > 128 && ceil_div(hx, 128) * ceil_div(hy, 256) >= 74) ? 256 : 128;  // narrow tiles while SMs would idle
     g.bk = 64;
     g.tiles = ceil_div(hx, 128) * ceil_div(hy, g.bn);
     min_blocks = 8;
