@@ -519,12 +519,16 @@ bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t
 
 int umma_rank_pad(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 
+// CTAs that share the rows of one 128-column tile of Z = Y^T X.  A CTA streams its rows at about one SM's
+// share of the HBM bandwidth whatever the grid, and every extra split costs a partial tile and a pass of the
+// finishing CTA over it, so the rows are split only while tiles alone leave SMs empty: about one CTA per SM,
+// at most 8 splits, at least 256 rows each (measured on 8 ... 512 tiles: best at 148 / tiles, rounded).
 int umma_cols_acc_splits(int S, int64_t N, int64_t h) {
   const int64_t tiles = ceil_div(h, 128) * S;
   const int64_t kb = ceil_div(N, 64);
-  int64_t splits = ceil_div(148 * 3, tiles);
-  if (splits > kb / 4) splits = kb / 4;  // at least 4 blocks (256 rows) per split
-  if (splits > 16) splits = 16;
+  int64_t splits = (148 + tiles / 2) / tiles;
+  if (splits > 8) splits = 8;
+  if (splits > kb / 4) splits = kb / 4;
   if (splits < 1) splits = 1;
   const int64_t per = ceil_div(kb, splits);
   return (int)ceil_div(kb, per);  // no empty split
