@@ -181,6 +181,20 @@ dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* 
                            float* grad, dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The same reconstruction (Algorithm 1, the P^T Q step) for `batch` layers of one shape in one go:
+ * entry b owns rows b*K .. b*K+K-1 of the stacks and the b-th h_in x h_out gradient,
+ *     grad[b][a][c] = sum_k Pcat[b*K + k][a] * Qcat[b*K + k][c].
+ * The entries are independent; batching only saves launches (a single reconstruction is a few
+ * microseconds of work).  Arguments, precision and errors as for dad_reconstruct; batch in 1 .. 65535;
+ * ws_bytes >= dad_reconstruct_batched_workspace_bytes(h_in, h_out, K, batch, math).  batch = 1 is
+ * dad_reconstruct itself, bit for bit.
+ */
+size_t dad_reconstruct_batched_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, int batch, dad_dtype math);
+dad_status dad_reconstruct_batched(int64_t h_in, int64_t h_out, int64_t K, int batch, const float* Pcat,
+                                   const float* Qcat, float* grad, dad_dtype math, void* ws, size_t ws_bytes,
+                                   void* cuda_stream);
+
+/*
  * The whole per-layer path from HOST memory (Algorithm 1 with the direct sum of outer products at the
  * aggregator): copies A, D (laid out by `layer`, but in host memory) and Q0 to the device, runs
  * dad_rank_compress -> dad_gather_factors -> dad_reconstruct there, and copies the h_in x h_out fp32 gradient

@@ -24,6 +24,7 @@ STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD
 # every symbol include/dad.h declares
 EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
            "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
+           "dad_reconstruct_batched_workspace_bytes", "dad_reconstruct_batched",
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
            "dad_rank_compress_gram",
@@ -76,6 +77,12 @@ def lib() -> ctypes.CDLL:
         L.dad_reconstruct.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, ctypes.c_int, vp,
                                       ctypes.c_size_t, vp]
         L.dad_reconstruct.restype = ctypes.c_int
+        L.dad_reconstruct_batched_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
+                                                              ctypes.c_int]
+        L.dad_reconstruct_batched_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_reconstruct_batched.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, vp, vp, vp,
+                                              ctypes.c_int, vp, ctypes.c_size_t, vp]
+        L.dad_reconstruct_batched.restype = ctypes.c_int
         L.dad_reconstruct_static.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, ctypes.c_int, vp]
         L.dad_reconstruct_static.restype = ctypes.c_int
         L.dad_aggregate_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int]
@@ -202,6 +209,18 @@ def dad_reconstruct(h_in: int, h_out: int, K: int, Pcat, Qcat, grad, math: int =
     _check(st, "dad_reconstruct")
 
 
+def dad_reconstruct_batched_workspace_bytes(h_in: int, h_out: int, K: int, batch: int, math: int) -> int:
+    return int(lib().dad_reconstruct_batched_workspace_bytes(h_in, h_out, K, batch, math))
+
+
+def dad_reconstruct_batched(h_in: int, h_out: int, K: int, batch: int, Pcat, Qcat, grad, math: int = DAD_F32, ws=None,
+                            stream=None):
+    """`batch` reconstructions of one shape in one go: entry b owns rows b*K .. b*K+K-1 of the stacks and grad[b]."""
+    st = lib().dad_reconstruct_batched(h_in, h_out, K, batch, _ptr(Pcat), _ptr(Qcat), _ptr(grad), math, _ptr(ws),
+                                       ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_reconstruct_batched")
+
+
 DAD_STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -291,7 +310,7 @@ class LayerPlan:
     `groups` > 1 stacks that many layers of the same shape in one plan: A and D then hold
     groups * S slices (layer g owns slices g*S .. g*S+S-1), the power iterations of all of them run
     in the same launches (slices are independent), and each layer is reconstructed from its own rows
-    of the stacks; `grad` is then groups x h_in x h_out."""
+    of the stacks (one batched call); `grad` is then groups x h_in x h_out."""
 
     def __init__(self, A: torch.Tensor, D: torch.Tensor, r: int, iters: int, zero_copy_gather: bool = False,
                  groups: int = 1):
@@ -317,15 +336,14 @@ class LayerPlan:
         if nws == 0:
             raise ValueError("invalid layer / rank / iteration count")
         self.K = self.sites * r
-        self.ws = new_workspace(max(nws, dad_reconstruct_workspace_bytes(L.h_in, L.h_out, self.K, self.math)), dev)
+        self.ws = new_workspace(max(nws, dad_reconstruct_batched_workspace_bytes(L.h_in, L.h_out, self.K, groups,
+                                                                                 self.math)), dev)
         self.bytes_tx = bytes_array(L.S)
 
     def step(self, A, D, Q0, stream=None):
         L = self.layer
         dad_rank_compress(L, A, D, self.r, self.iters, Q0, self.P, self.Q, self.sigma, self.ws, stream)
         dad_gather_factors(L, self.r, self.P, self.Q, self.Pcat, self.Qcat, self.bytes_tx, stream)
-        for g in range(self.groups):
-            rows = slice(g * self.K, (g + 1) * self.K)
-            dad_reconstruct(L.h_in, L.h_out, self.K, self.Pcat[rows], self.Qcat[rows], self.grads[g], self.math,
-                            self.ws, stream)
+        dad_reconstruct_batched(L.h_in, L.h_out, self.K, self.groups, self.Pcat, self.Qcat, self.grads, self.math,
+                                self.ws, stream)
         return self.grad

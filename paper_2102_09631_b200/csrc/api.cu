@@ -91,14 +91,14 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc) {
   return w;
 }
 
-GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands) {
+GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands, int batch) {
   GemmWs w;
   memset(&w, 0, sizeof(w));
   size_t off = 0;
   w.status = off;
   off += 256;
-  const GemmPlan g = umma_gemm_plan(hx, hy, S, N);
-  const size_t tiles = (size_t)g.tiles;
+  const GemmPlan g = umma_gemm_plan(hx, hy, S, N, batch);
+  const size_t tiles = (size_t)g.tiles * (size_t)batch;
   w.n_counters = tiles;
   w.counters = off;
   off = align_up(off + tiles * sizeof(unsigned), 256);
@@ -107,9 +107,9 @@ GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_ope
   w.Xb = w.Yb = off;
   if (convert_operands) {
     w.Xb = off;
-    off = align_up(off + (size_t)S * N * hx * 2, 256);
+    off = align_up(off + (size_t)batch * S * N * hx * 2, 256);
     w.Yb = off;
-    off = align_up(off + (size_t)S * N * hy * 2, 256);
+    off = align_up(off + (size_t)batch * S * N * hy * 2, 256);
   }
   w.total = off;
   return w;
@@ -237,14 +237,15 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
 
 static cudaError_t run_gemm_tc(const void* X, int64_t ldX, int64_t strideX, const void* Y, int64_t ldY, int64_t strideY,
                                int S, int64_t N, int64_t hx, int64_t hy, float* C, char* ws, const GemmWs& w,
-                               cudaStream_t st) {
+                               cudaStream_t st, int batch = 1) {
   // the second status slot (byte 4) belongs to the dense products; the first keeps what a compress call reported
   cudaError_t err = cudaMemsetAsync(ws + w.status + 4, 0, w.counters + w.n_counters * sizeof(unsigned) - w.status - 4, st);
   if (err != cudaSuccess) return err;
   CUtensorMap tmX, tmY;
-  const GemmPlan g = umma_gemm_plan(hx, hy, S, N);
-  if (!make_tmap_bf16_3d(&tmX, X, hx, N, S, (uint64_t)ldX * 2, (uint64_t)strideX * 2, 64, (uint32_t)g.bk) ||
-      !make_tmap_bf16_3d(&tmY, Y, hy, N, S, (uint64_t)ldY * 2, (uint64_t)strideY * 2, 64, (uint32_t)g.bk))
+  const GemmPlan g = umma_gemm_plan(hx, hy, S, N, batch);
+  const uint64_t d2 = batch > 1 ? (uint64_t)batch : (uint64_t)S;  // third dimension: sites of one product, or products
+  if (!make_tmap_bf16_3d(&tmX, X, hx, N, d2, (uint64_t)ldX * 2, (uint64_t)strideX * 2, 64, (uint32_t)g.bk) ||
+      !make_tmap_bf16_3d(&tmY, Y, hy, N, d2, (uint64_t)ldY * 2, (uint64_t)strideY * 2, 64, (uint32_t)g.bk))
     return cudaErrorInvalidValue;
   return umma_gemm_tn(tmX, tmY, g, hx, hy, C, reinterpret_cast<float*>(ws + w.partial),
                       reinterpret_cast<unsigned*>(ws + w.counters), reinterpret_cast<int*>(ws + w.status + 4), st);
@@ -357,34 +358,48 @@ static bool reconstruct_tc(int64_t h_in, int64_t h_out, int64_t K, dad_dtype mat
   return math == DAD_BF16 && h_in % 8 == 0 && h_out % 8 == 0 && 3 * K <= 0x7fffffff && tmap_encoder_available();
 }
 
-size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
-  if (h_in < 1 || h_out < 1 || K < 1) return 0;
+size_t dad_reconstruct_batched_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, int batch, dad_dtype math) {
+  if (h_in < 1 || h_out < 1 || K < 1 || batch < 1) return 0;
   if (!reconstruct_tc(h_in, h_out, K, math)) return 0;
-  return gemm_ws_layout(h_in, h_out, 1, 3 * K, true).total;
+  return gemm_ws_layout(h_in, h_out, 1, 3 * K, true, batch).total;
 }
 
-dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat, float* grad,
-                           dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream) {
-  if (h_in < 1 || h_out < 1 || K < 1 || h_in > 0x7fffffff || h_out > 0x7fffffff) return DAD_ERR_SHAPE;
+size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
+  return dad_reconstruct_batched_workspace_bytes(h_in, h_out, K, 1, math);
+}
+
+dad_status dad_reconstruct_batched(int64_t h_in, int64_t h_out, int64_t K, int batch, const float* Pcat,
+                                   const float* Qcat, float* grad, dad_dtype math, void* ws, size_t ws_bytes,
+                                   void* cuda_stream) {
+  if (h_in < 1 || h_out < 1 || K < 1 || h_in > 0x7fffffff || h_out > 0x7fffffff || batch < 1 || batch > 65535)
+    return DAD_ERR_SHAPE;
   if (math != DAD_F32 && math != DAD_BF16) return DAD_ERR_DTYPE;
   if (!Pcat || !Qcat || !grad) return DAD_ERR_NULL;
   if (!aligned(Pcat, 16) || !aligned(Qcat, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  cudaError_t err;
+  cudaError_t err = cudaSuccess;
   if (reconstruct_tc(h_in, h_out, K, math)) {
-    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, 3 * K, true);  // three bf16 products, one contraction
+    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, 3 * K, true, batch);  // three bf16 products, one contraction
     if (!ws) return DAD_ERR_NULL;
     if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
     if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
     __nv_bfloat16* Xb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Xb);
     __nv_bfloat16* Yb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Yb);
-    err = stack_split3(Pcat, (size_t)K * h_in, Xb, Qcat, (size_t)K * h_out, Yb, st);
+    err = stack_split3(Pcat, (size_t)K * h_in, Xb, Qcat, (size_t)K * h_out, Yb, batch, st);
     if (err == cudaSuccess)
-      err = run_gemm_tc(Xb, h_in, 3 * K * h_in, Yb, h_out, 3 * K * h_out, 1, 3 * K, h_in, h_out, grad, (char*)ws, w, st);
+      err = run_gemm_tc(Xb, h_in, 3 * K * h_in, Yb, h_out, 3 * K * h_out, 1, 3 * K, h_in, h_out, grad, (char*)ws, w, st,
+                        batch);
   } else {
-    err = gemm_tn_simt(DAD_F32, Pcat, h_in, 0, Qcat, h_out, 0, 1, K, h_in, h_out, grad, st);
+    for (int b = 0; b < batch && err == cudaSuccess; ++b)
+      err = gemm_tn_simt(DAD_F32, Pcat + (size_t)b * K * h_in, h_in, 0, Qcat + (size_t)b * K * h_out, h_out, 0, 1, K, h_in,
+                         h_out, grad + (size_t)b * h_in * h_out, st);
   }
   return err == cudaSuccess ? DAD_OK : DAD_ERR_CUDA;
+}
+
+dad_status dad_reconstruct(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat, const float* Qcat, float* grad,
+                           dad_dtype math, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return dad_reconstruct_batched(h_in, h_out, K, 1, Pcat, Qcat, grad, math, ws, ws_bytes, cuda_stream);
 }
 
 dad_status dad_check(const void* ws, void* cuda_stream) {

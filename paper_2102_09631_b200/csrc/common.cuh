@@ -75,7 +75,7 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc);
 struct GemmWs {
   size_t status, counters, n_counters, partial, Xb, Yb, total;  // Xb/Yb: bf16 copies of fp32 operands
 };
-GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands);
+GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands, int batch = 1);
 
 // Whether the tensor-core kernels take this layer: bf16, all extents and strides multiples of 8
 // elements (TMA wants 16-byte strides), and the driver's tensor-map encoder is available.
@@ -120,8 +120,9 @@ cudaError_t row_norms(const T* M, int64_t rows, int64_t h, float* out, cudaStrea
 // planes[s][0/1][j][c] = hi / lo bf16 terms of in[s][j][c]  (j < r; plane_rows >= r rows per plane)
 cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16* planes, int plane_rows,
                          cudaStream_t st);
+// Three-term bf16 operand stacks of `batch` reconstructions: P is batch x (nP elements), X3 is batch x 3 x nP, same for Q.
 cudaError_t stack_split3(const float* P, size_t nP, __nv_bfloat16* X3, const float* Q, size_t nQ, __nv_bfloat16* Y3,
-                         cudaStream_t st);
+                         int batch, cudaStream_t st);
 
 // ---- tensor-core launchers (umma_gemm.cu) -------------------------------------------------------
 bool tmap_encoder_available();
@@ -132,10 +133,11 @@ int umma_cols_acc_splits(int S, int64_t N, int64_t h);
 // Geometry of the dense product C = X^T Y (hx x hy, contraction over S sites of N rows): tile bm x bn, stages of
 // bk contraction rows (the row count of the operands' TMA boxes), `splits` CTAs share a tile's contraction.
 struct GemmPlan {
-  int bm, bn, bk, splits;
-  int64_t tiles, k_blocks, kb_per_site;
+  int bm, bn, bk, splits, batch;
+  int64_t tiles, k_blocks, kb_per_site;  // tiles: per batch entry
 };
-GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N);
+// batch > 1: that many independent products of one site each (S must be 1) in one launch.
+GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch);
 cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S, int64_t N, int64_t h, int r,
                           __nv_bfloat16* yt_planes, int64_t ld_planes, int* status, cudaStream_t st);
 cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,

@@ -147,15 +147,19 @@ cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16
 // fp32-level accuracy: with x = hi(x) + lo(x) (two bf16 terms), P^T Q ~= hi^T hi + hi^T lo + lo^T hi, the
 // dropped lo^T lo term being 2^-16 relative.  The three products become one contraction of length 3K over
 //     X3 = [hi(P); hi(P); lo(P)]   and   Y3 = [hi(Q); lo(Q); hi(Q)].
-// Four elements per thread; nP and nQ are multiples of 4 and all pointers 8-byte aligned.
+// Four elements per thread; nP and nQ are multiples of 4 and all pointers 8-byte aligned.  `batch` independent
+// factor stacks lie one after the other in P and Q; each gets its own three-term stack in X3 and Y3.
 __global__ void stack_split3_kernel(const float* __restrict__ P, size_t nP, __nv_bfloat16* __restrict__ X3,
-                                    const float* __restrict__ Q, size_t nQ, __nv_bfloat16* __restrict__ Y3) {
+                                    const float* __restrict__ Q, size_t nQ, __nv_bfloat16* __restrict__ Y3, int batch) {
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   const size_t qP = nP / 4, qQ = nQ / 4;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < qP + qQ; i += stride) {
-    const bool isP = i < qP;
-    const size_t q = isP ? i : i - qP;
-    const float4 v = reinterpret_cast<const float4*>(isP ? P : Q)[q];
+  const size_t allP = qP * (size_t)batch, all = (qP + qQ) * (size_t)batch;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < all; i += stride) {
+    const bool isP = i < allP;
+    const size_t lin = isP ? i : i - allP;     // quad index over all batch entries of this operand
+    const size_t plane = isP ? qP : qQ;        // quads per term of one batch entry
+    const size_t b = lin / plane, q = lin % plane;
+    const float4 v = reinterpret_cast<const float4*>(isP ? P : Q)[lin];
     const float f[4] = {v.x, v.y, v.z, v.w};
     __align__(8) __nv_bfloat16 hi[4], lo[4];
 #pragma unroll
@@ -164,8 +168,7 @@ __global__ void stack_split3_kernel(const float* __restrict__ P, size_t nP, __nv
       lo[u] = __float2bfloat16_rn(f[u] - __bfloat162float(hi[u]));
     }
     const uint2 h2 = *reinterpret_cast<const uint2*>(hi), l2 = *reinterpret_cast<const uint2*>(lo);
-    uint2* out = reinterpret_cast<uint2*>(isP ? X3 : Y3);
-    const size_t plane = isP ? qP : qQ;
+    uint2* out = reinterpret_cast<uint2*>(isP ? X3 : Y3) + b * 3 * plane;
     out[q] = h2;
     out[plane + q] = isP ? h2 : l2;
     out[2 * plane + q] = isP ? l2 : h2;
@@ -173,12 +176,12 @@ __global__ void stack_split3_kernel(const float* __restrict__ P, size_t nP, __nv
 }
 
 cudaError_t stack_split3(const float* P, size_t nP, __nv_bfloat16* X3, const float* Q, size_t nQ, __nv_bfloat16* Y3,
-                         cudaStream_t st) {
+                         int batch, cudaStream_t st) {
   cudaError_t err = cudaSuccess;
-  size_t blocks = ((nP + nQ) / 4 + 255) / 256;
+  size_t blocks = ((nP + nQ) / 4 * (size_t)batch + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  DAD_LAUNCH(err, "stack_split3", stack_split3_kernel, (unsigned)blocks, 256, 0, st, P, nP, X3, Q, nQ, Y3);
+  DAD_LAUNCH(err, "stack_split3", stack_split3_kernel, (unsigned)blocks, 256, 0, st, P, nP, X3, Q, nQ, Y3, batch);
   return err;
 }
 

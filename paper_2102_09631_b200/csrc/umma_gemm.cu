@@ -44,6 +44,7 @@ struct UmmaParams {
   float* out_f32;    // EPI_Z: [batch][r][ld_out];  EPI_C: [m][ld_out]
   float* out2_f32;   // EPI_Z: optional second copy, same layout
   int64_t ld_out;
+  int64_t out_batch_stride;   // EPI_C: elements between the outputs of consecutive batch entries
   __nv_bfloat16* out_planes;  // EPI_YT / EPI_Z: [batch][2][plane_rows][ld_planes] (hi plane, lo plane), or null
   int64_t ld_planes;
   int plane_rows;    // rows per plane (r rounded up to the MMA width); rows >= r are never written
@@ -240,7 +241,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         if (gm < p.m_extent) {
           if constexpr (EPI == EPI_C) {
-            float* dst = p.out_f32 + gm * p.ld_out + n0 + c * 16;
+            float* dst = p.out_f32 + (int64_t)batch * p.out_batch_stride + gm * p.ld_out + n0 + c * 16;
             if (n0 + c * 16 + 16 <= p.n_extent && (p.ld_out & 3) == 0) {
 #pragma unroll
               for (int i = 0; i < 4; ++i)
@@ -614,9 +615,9 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
 // the 256 x 256 two-accumulator kernel; everything else 128 x BN tiles, BN = 256 where the output is wide
 // enough (a 128 x 128 x 16 MMA needs 128 B/clk of operands from shared memory, a 128 x 256 x 16 one
 // 96 B/clk).  Splits of the contraction fill the 148 SMs when the tiles alone do not.
-GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N) {
+GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch) {
   GemmPlan g;
-  const bool big = hx >= 256 && hy >= 256 && N * S >= kGemm256MinRows;
+  const bool big = batch == 1 && hx >= 256 && hy >= 256 && N * S >= kGemm256MinRows;
   int64_t min_blocks;
   if (big) {
     g.bm = 256;
@@ -626,14 +627,15 @@ GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N) {
     min_blocks = 512 / g.bk;
   } else {
     g.bm = 128;
-    g.bn = (hy > 128 && ceil_div(hx, 128) * ceil_div(hy, 256) >= 74) ? 256 : 128;  // narrow tiles while SMs would idle
+    g.bn = (hy > 128 && ceil_div(hx, 128) * ceil_div(hy, 256) * batch >= 74) ? 256 : 128;  // narrow tiles while SMs would idle
     g.bk = 64;
     g.tiles = ceil_div(hx, 128) * ceil_div(hy, g.bn);
     min_blocks = 8;
   }
   g.kb_per_site = ceil_div(N, g.bk);
   g.k_blocks = g.kb_per_site * S;
-  int64_t splits = 148 / g.tiles;
+  g.batch = batch;
+  int64_t splits = 148 / (g.tiles * batch);
   if (splits > g.k_blocks / min_blocks) splits = g.k_blocks / min_blocks;
   if (splits > 32) splits = 32;
   if (splits < 1) splits = 1;
@@ -668,21 +670,23 @@ static cudaError_t launch_gemm256(const CUtensorMap& tmA, const CUtensorMap& tmB
 }
 
 // C (hx x hy, fp32) <- sum over sites and rows of X^T Y.  tmX: (hx, N, S), tmY: (hy, N, S), boxes 64 x plan.bk.
+// With plan.batch > 1 (and S = 1) the third tensor dimension counts independent products instead: C is batch x hx x hy.
 cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& g, int64_t hx, int64_t hy,
                          float* C, float* partial, unsigned* counters, int* status, cudaStream_t st) {
   UmmaParams p{};
   p.m_extent = (int)hx;
   p.n_extent = (int)hy;
-  p.kb_per_site = (int)g.kb_per_site;
+  p.kb_per_site = g.batch > 1 ? 0 : (int)g.kb_per_site;  // batched: one site per entry, the entry from blockIdx.z
   p.k_blocks = (int)g.k_blocks;
   p.splits = g.splits;
   p.kb_per_split = (int)ceil_div(g.k_blocks, g.splits);
   p.out_f32 = C;
   p.ld_out = hy;
+  p.out_batch_stride = hx * hy;
   p.partial = partial;
   p.counters = counters;
   p.status = status;
-  dim3 grid((unsigned)ceil_div(hx, g.bm), (unsigned)(ceil_div(hy, g.bn) * g.splits), 1);
+  dim3 grid((unsigned)ceil_div(hx, g.bm), (unsigned)(ceil_div(hy, g.bn) * g.splits), (unsigned)g.batch);
   if (g.bm == 256) {
     cudaError_t err = launch_gemm256<kGemm256BK, kGemm256Stages>(tmX, tmY, p, grid, st);
     if (err != cudaSuccess || g.splits == 1) return err;

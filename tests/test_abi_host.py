@@ -101,6 +101,9 @@ def test_bad_arguments_are_rejected_before_any_launch(B):
     assert lib.dad_reconstruct(0, 4, 4, p, p, p, 0, null, 0, None) == E["DAD_ERR_SHAPE"]
     assert lib.dad_reconstruct(4, 4, 4, p, null, p, 0, null, 0, None) == E["DAD_ERR_NULL"]
     assert lib.dad_reconstruct(4, 4, 4, p, p, p, 9, null, 0, None) == E["DAD_ERR_DTYPE"]
+    assert lib.dad_reconstruct_batched(4, 4, 4, 0, p, p, p, 0, null, 0, None) == E["DAD_ERR_SHAPE"]
+    assert lib.dad_reconstruct_batched(4, 4, 4, 2, p, p, null, 0, null, 0, None) == E["DAD_ERR_NULL"]
+    assert lib.dad_reconstruct_batched_workspace_bytes(4, 4, 4, 0, 1) == 0
     assert lib.dad_gather_factors(ctypes.byref(L), 0, p, p, p, p, None, None) == E["DAD_ERR_RANK"]
     assert lib.dad_check(null, None) == E["DAD_ERR_NULL"]
     assert B.dad_launch_count() == before

@@ -154,6 +154,29 @@ def test_full_grad_long_contraction(oracle, B, S, N, h_in, h_out):
     assert rel(grads[0].double().numpy(), oracle.full_grad(A, D)) <= 1e-4
 
 
+@pytest.mark.parametrize("h_in,h_out,K,batch", [(1024, 1024, 256, 16), (264, 520, 40, 3), (70, 50, 12, 2)])
+def test_reconstruct_batched_is_the_per_layer_sum_of_outer_products(oracle, B, h_in, h_out, K, batch):
+    """Algorithm 1's P^T Q step for several layers of one shape in one call: every entry against the oracle's
+    sum of outer products over its own K rows of the stacks, and batch = 1 against dad_reconstruct bit for bit."""
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(1000 + K)
+    Pcat = torch.randn(batch * K, h_in, generator=g)
+    Qcat = torch.randn(batch * K, h_out, generator=g)
+    for math, tol in ((B.DAD_F32, 1e-5), (B.DAD_BF16, 1e-4)):
+        ws = B.new_workspace(B.dad_reconstruct_batched_workspace_bytes(h_in, h_out, K, batch, math), dev)
+        grads = torch.full((batch, h_in, h_out), float("nan"), device=dev)
+        B.dad_reconstruct_batched(h_in, h_out, K, batch, Pcat.to(dev), Qcat.to(dev), grads, math, ws)
+        B.dad_check(ws)
+        for b in range(batch):
+            rows = slice(b * K, (b + 1) * K)
+            ref = oracle.reconstruct(Pcat[rows], Qcat[rows])
+            assert rel(grads[b].double().cpu().numpy(), ref) <= tol, (b, math)
+        one, single = torch.empty(h_in, h_out, device=dev), torch.empty(h_in, h_out, device=dev)
+        B.dad_reconstruct_batched(h_in, h_out, K, 1, Pcat.to(dev), Qcat.to(dev), one, math, ws)
+        B.dad_reconstruct(h_in, h_out, K, Pcat.to(dev), Qcat.to(dev), single, math, ws)
+        assert torch.equal(one, single)
+
+
 def test_factors_match_on_separated_spectrum(oracle, B):
     """With well separated singular values and enough iterations each vector is determined up to
     rounding (thin QR with positive diagonal fixes the sign), so the raw factors agree too."""
