@@ -580,7 +580,7 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
   switch (umma_rank_pad(r)) {
     case 16: return launch_umma<16, false, false, 2, EPI_YT, 5>(tmX, tmF, p, grid, "rows_dot_tc", st);
     case 32: return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
-    default: return launch_umma<64, false, false, 2, EPI_YT, 3>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    default: return launch_umma<64, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
   }
 }
 
