@@ -161,11 +161,9 @@ static cudaError_t run_compress(const dad_layer& L, const void* A, const void* D
     DAD_STEP(cols_acc<TAcc>(L.dtype, D, L.ldD, L.strideD, S, N, ho, Y, r, G, nullptr, part, ctr_cols, st));  // Gt = W^T D
     // the second pass returns at once for sites whose first pass was well conditioned, so both write the outputs
     float* q32 = (f64 && k == iters - 1) ? Q : nullptr;
-    if constexpr (!f64) {
-      if (orth_cluster_fits(r, ho)) {
-        DAD_STEP(orth_cluster(reinterpret_cast<float*>(G), S, r, ho, tol, status, nullptr, nullptr, 0, st));
-        continue;
-      }
+    if (orth_cluster_fits(r, ho, sizeof(TAcc))) {
+      DAD_STEP(orth_cluster<TAcc>(G, S, r, ho, tol, status, q32, nullptr, 0, st));
+      continue;
     }
     DAD_STEP(cholqr_pass<TAcc>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,
                                nullptr, 0, st));

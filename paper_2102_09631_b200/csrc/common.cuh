@@ -102,9 +102,10 @@ cudaError_t cholqr_pass(T* G, int S, int r, int64_t h, int pass, double tol, dou
                         int* status, float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
 
 // The same orthonormalisation (both passes, second one decided on the device) in one launch, for
-// fp32 storage: a thread-block cluster per site keeps the vectors in shared memory throughout.
-bool orth_cluster_fits(int r, int64_t h);
-cudaError_t orth_cluster(float* G, int S, int r, int64_t h, double tol, int* status, float* out32,
+// fp32 or fp64 storage (T): a thread-block cluster per site keeps the vectors in shared memory throughout.
+bool orth_cluster_fits(int r, int64_t h, size_t elem_bytes = 4);
+template <typename T>
+cudaError_t orth_cluster(T* G, int S, int r, int64_t h, double tol, int* status, float* out32,
                          __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
 
 // C[a][b] = sum_{s,n} X[s][n][a] * Y[s][n][b]  (fp32 FMA), C: hx x hy fp32 contiguous

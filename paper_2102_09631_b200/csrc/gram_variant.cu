@@ -160,6 +160,10 @@ dad_status dad_rank_compress_gram(const dad_layer* L, const void* A, const void*
     if (err != cudaSuccess) return DAD_ERR_CUDA;
     DAD_STEP(cols_acc<double>(DAD_F32, D, L->ldD, L->strideD, S, N, ho, T, r, G, nullptr, part, ctr_cols, st));  // D^T (C v)
     float* q32 = (k == iters - 1) ? Q : nullptr;
+    if (orth_cluster_fits(r, ho, sizeof(double))) {
+      DAD_STEP(orth_cluster<double>(G, S, r, ho, tol, status, q32, nullptr, 0, st));
+      continue;
+    }
     DAD_STEP(cholqr_pass<double>(G, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,
                                  nullptr, 0, st));
     DAD_STEP(cholqr_pass<double>(G, S, r, ho, 1, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, q32,

@@ -1,4 +1,5 @@
-// Orthonormalisation of the r iterate vectors of a site in ONE launch (fp32 storage pipeline):
+// Orthonormalisation of the r iterate vectors of a site in ONE launch (vectors stored as fp32, or as fp64 in
+// the pipeline of fp32 inputs):
 // a thread-block cluster of C CTAs per site, each holding a slab of r x W columns in shared
 // memory for the whole Cholesky-QR (both passes), so the vectors are read from and written to
 // global memory exactly once.
@@ -24,7 +25,13 @@ namespace dad {
 
 namespace {
 constexpr double kPivotFloor = 1e-14;          // (1e-7)^2 of the squared length
-constexpr double kSecondPassBelowSq = 1e-10;   // (1e-5)^2: ratio of squared lengths that asks for a second pass
+// Ratio of squared lengths R_jj^2 / ||g_j||^2 below which a second pass is asked for: (1e-5)^2 for fp32 storage (one
+// fp64 pass leaves a defect of 1e-16 cond^2 <= 1e-6, the level of the storage), (1e-3)^2 for fp64 storage (<= 1e-10).
+template <typename T>
+constexpr double second_pass_below_sq() { return sizeof(T) == 4 ? 1e-10 : 1e-6; }
+template <typename T> struct Vec2;
+template <> struct Vec2<float> { using type = float2; };
+template <> struct Vec2<double> { using type = double2; };
 constexpr int kThreads = 256;
 
 struct OrthGeom {
@@ -33,23 +40,23 @@ struct OrthGeom {
   int Wp;       // padded row length of the slab in floats
   int nblocks;  // lower-triangular register blocks of the Gram matrix
   int cgs;      // column groups the slab is split into for the Gram phase
-  size_t off_gram, off_L, off_vec, total;  // byte offsets after the slab
+  size_t off_gram, off_L, off_vec, total;  // byte offsets after the slab (of elements of `esize` bytes)
 };
 
 template <int BS>
-__host__ __device__ inline OrthGeom orth_geom(int r, int64_t h, int C) {
+__host__ __device__ inline OrthGeom orth_geom(int r, int64_t h, int C, size_t esize) {
   OrthGeom g;
   constexpr int RB = BS < 4 ? 4 : BS;
   g.rp = (r + RB - 1) / RB * RB;
   int W = (int)((h + C - 1) / C);
   g.W = (W + 3) / 4 * 4;
-  g.Wp = g.W + 2;  // even (float2 accesses), and rows 8 apart do not share a bank
+  g.Wp = g.W + 2;  // even (two-element vector accesses), and rows 8 apart do not share a bank
   const int nb = g.rp / BS;
   g.nblocks = nb * (nb + 1) / 2;
   g.cgs = kThreads / g.nblocks;
   if (g.cgs < 1) g.cgs = 1;
   if (g.cgs > 8) g.cgs = 8;
-  size_t off = sizeof(float) * (size_t)g.rp * g.Wp;
+  size_t off = esize * (size_t)g.rp * g.Wp;
   off = (off + 15) / 16 * 16;
   g.off_gram = off;  // this CTA's partial Gram, rp x rp doubles (read by the other CTAs of the cluster)
   off += sizeof(double) * (size_t)g.rp * g.rp;
@@ -62,15 +69,15 @@ __host__ __device__ inline OrthGeom orth_geom(int r, int64_t h, int C) {
 }
 
 template <int BS>
-inline bool slab_fits(int r, int64_t h, int C) { return orth_geom<BS>(r, h, C).total <= 200 * 1024; }
+inline bool slab_fits(int r, int64_t h, int C, size_t esize) { return orth_geom<BS>(r, h, C, esize).total <= 200 * 1024; }
 
 // CTAs per site.  Every CTA of a cluster repeats the r x r factorisation, so the cluster is kept as small as
 // still fills the GPU with S sites (and as the slab of h / C columns allows); with few sites it grows to 8.
-inline int cluster_size_for(int r, int64_t h, int S) {
+inline int cluster_size_for(int r, int64_t h, int S, size_t esize) {
   int best = 0;
   for (int C = 1; C <= 8; C *= 2) {
     if (C > 1 && h / C < 128) break;
-    const bool fits = r >= 32 ? slab_fits<8>(r, h, C) : slab_fits<2>(r, h, C);
+    const bool fits = r >= 32 ? slab_fits<8>(r, h, C, esize) : slab_fits<2>(r, h, C, esize);
     if (!fits) continue;
     best = C;
     if ((int64_t)S * C >= 2 * 148) break;
@@ -79,14 +86,16 @@ inline int cluster_size_for(int r, int64_t h, int S) {
 }
 }  // namespace
 
-template <int BS>
+template <int BS, typename T>
 __global__ void __launch_bounds__(kThreads)
-orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, int* __restrict__ status,
+orth_cluster_kernel(T* __restrict__ G, int r, int64_t h, int C, double tol, int* __restrict__ status,
                     float* __restrict__ out32, __nv_bfloat16* __restrict__ planes, int plane_rows) {
+  using T2 = typename Vec2<T>::type;
+  constexpr bool kF32 = sizeof(T) == 4;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
-  const OrthGeom g = orth_geom<BS>(r, h, C);
-  float* slab = reinterpret_cast<float*>(smem_raw);
+  const OrthGeom g = orth_geom<BS>(r, h, C, sizeof(T));
+  T* slab = reinterpret_cast<T*>(smem_raw);
   double* gram = reinterpret_cast<double*>(smem_raw + g.off_gram);
   double* Lm = reinterpret_cast<double*>(smem_raw + g.off_L);
   double* diag0 = reinterpret_cast<double*>(smem_raw + g.off_vec);
@@ -101,7 +110,7 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   const int rank = (int)cluster.block_rank();
   const int rp = g.rp, W = g.W, Wp = g.Wp, LR = rp + 1;
   const int64_t c0 = (int64_t)rank * W;
-  float* Gs = G + (int64_t)s * r * h;
+  T* Gs = G + (int64_t)s * r * h;
   const double tol2 = tol * tol;
 
   // the next kernel in the stream may begin its set-up now; it waits for this grid before touching memory
@@ -109,7 +118,9 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
 
   // ---- load the slab (rows >= r and columns >= h are zero) ----
   // Loads are issued eight at a time per thread before any is stored, so that their latencies overlap.
-  if ((h & 3) == 0) {
+  if (kF32 && (h & 3) == 0) {
+    const float* Gf = reinterpret_cast<const float*>(Gs);
+    float* slabf = reinterpret_cast<float*>(slab);
     const int W4 = W / 4, total = rp * W4;
     for (int base = 0; base < total; base += kThreads * 8) {
       float4 v[8];
@@ -118,13 +129,13 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
         const int idx = base + u * kThreads + tid;
         const int j = idx / W4, c = (idx % W4) * 4;
         v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (idx < total && j < r && c0 + c < h) v[u] = *reinterpret_cast<const float4*>(Gs + (int64_t)j * h + c0 + c);
+        if (idx < total && j < r && c0 + c < h) v[u] = *reinterpret_cast<const float4*>(Gf + (int64_t)j * h + c0 + c);
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int idx = base + u * kThreads + tid;
         if (idx < total) {
-          float* dst = slab + (idx / W4) * Wp + (idx % W4) * 4;  // 8-byte aligned (Wp is even)
+          float* dst = slabf + (idx / W4) * Wp + (idx % W4) * 4;  // 8-byte aligned (Wp is even)
           *reinterpret_cast<float2*>(dst) = make_float2(v[u].x, v[u].y);
           *reinterpret_cast<float2*>(dst + 2) = make_float2(v[u].z, v[u].w);
         }
@@ -133,12 +144,12 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   } else {
     const int total = rp * W;
     for (int base = 0; base < total; base += kThreads * 8) {
-      float v[8];
+      T v[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int idx = base + u * kThreads + tid;
         const int j = idx / W, c = idx % W;
-        v[u] = (idx < total && j < r && c0 + c < h) ? Gs[(int64_t)j * h + c0 + c] : 0.f;
+        v[u] = (idx < total && j < r && c0 + c < h) ? Gs[(int64_t)j * h + c0 + c] : T(0);
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
@@ -172,8 +183,8 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
           while ((bi + 1) * (bi + 2) / 2 <= b) ++bi;  // block row: bi(bi+1)/2 <= b
           bj = b - bi * (bi + 1) / 2;
           const int cbeg = grp * Wc, cend = (cbeg + Wc < W) ? cbeg + Wc : W;
-          const float* ra = slab + (bi * BS) * Wp;
-          const float* rb = slab + (bj * BS) * Wp;
+          const T* ra = slab + (bi * BS) * Wp;
+          const T* rb = slab + (bj * BS) * Wp;
           for (int c = cbeg; c < cend; ++c) {
             double a[BS], bb[BS];
 #pragma unroll
@@ -265,7 +276,7 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
           if (pass == 0) {
             piv1[j] = is_dead ? 0.0 : piv;
             orig1[j] = orig;
-            if (!is_dead && piv < kSecondPassBelowSq * orig) need2_s = 1;
+            if (!is_dead && piv < second_pass_below_sq<T>() * orig) need2_s = 1;
           }
           if (is_dead) dead_row[j] = 1;
           Lm[j * LR + j] = piv * il;
@@ -284,12 +295,12 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
         double v[4][2];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const float2 x = *reinterpret_cast<const float2*>(slab + (j0 + u) * Wp + c);
+          const T2 x = *reinterpret_cast<const T2*>(slab + (j0 + u) * Wp + c);
           v[u][0] = (double)x.x;
           v[u][1] = (double)x.y;
         }
         for (int l = 0; l < j0; ++l) {
-          const float2 q = *reinterpret_cast<const float2*>(slab + l * Wp + c);
+          const T2 q = *reinterpret_cast<const T2*>(slab + l * Wp + c);
           const double q0 = (double)q.x, q1 = (double)q.y;
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -302,9 +313,12 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
         for (int u = 0; u < 4; ++u) {
           const int j = j0 + u;
           const double il = dead_row[j] ? 0.0 : inv_l[j];
-          // the value stored (and used by the rows below) is the fp32-rounded one
-          const float o0 = (float)(v[u][0] * il), o1 = (float)(v[u][1] * il);
-          *reinterpret_cast<float2*>(slab + j * Wp + c) = make_float2(o0, o1);
+          // the value stored (and used by the rows below) is the one rounded to the storage type
+          const T o0 = (T)(v[u][0] * il), o1 = (T)(v[u][1] * il);
+          T2 o;
+          o.x = o0;
+          o.y = o1;
+          *reinterpret_cast<T2*>(slab + j * Wp + c) = o;
 #pragma unroll
           for (int w = u + 1; w < 4; ++w) {
             const double a = Lm[(j0 + w) * LR + j];
@@ -319,16 +333,18 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   }
 
   // ---- write the orthonormal vectors (and their bf16 hi/lo planes) ----
-  if ((h & 3) == 0) {
+  if (kF32 && (h & 3) == 0) {
+    float* Gf = reinterpret_cast<float*>(Gs);
+    const float* slabf = reinterpret_cast<const float*>(slab);
     const int W4 = W / 4;
     for (int idx = tid; idx < r * W4; idx += kThreads) {
       const int j = idx / W4, c = (idx % W4) * 4;
       const int64_t col = c0 + c;
       if (col < h) {
-        const float2 lo2 = *reinterpret_cast<const float2*>(slab + j * Wp + c);
-        const float2 hi2 = *reinterpret_cast<const float2*>(slab + j * Wp + c + 2);
+        const float2 lo2 = *reinterpret_cast<const float2*>(slabf + j * Wp + c);
+        const float2 hi2 = *reinterpret_cast<const float2*>(slabf + j * Wp + c + 2);
         const float f[4] = {lo2.x, lo2.y, hi2.x, hi2.y};
-        *reinterpret_cast<float4*>(Gs + (int64_t)j * h + col) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4*>(Gf + (int64_t)j * h + col) = make_float4(f[0], f[1], f[2], f[3]);
         if (out32) *reinterpret_cast<float4*>(out32 + ((int64_t)s * r + j) * h + col) = make_float4(f[0], f[1], f[2], f[3]);
         if (planes) {
           __nv_bfloat16 hi[4], lo[4];
@@ -348,9 +364,10 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
     for (int idx = tid; idx < r * W; idx += kThreads) {
       const int j = idx / W, c = idx % W;
       if (c0 + c < h) {
-        const float f = slab[j * Wp + c];
+        const T g_out = slab[j * Wp + c];
+        const float f = (float)g_out;
         const int64_t col = c0 + c;
-        Gs[(int64_t)j * h + col] = f;
+        Gs[(int64_t)j * h + col] = g_out;
         if (out32) out32[((int64_t)s * r + j) * h + col] = f;
         if (planes) {
           const __nv_bfloat16 hi = __float2bfloat16_rn(f);
@@ -362,10 +379,10 @@ orth_cluster_kernel(float* __restrict__ G, int r, int64_t h, int C, double tol, 
   }
 }
 
-template <int BS>
-static cudaError_t launch_orth_cluster(float* G, int S, int r, int64_t h, int C, double tol, int* status, float* out32,
+template <int BS, typename T>
+static cudaError_t launch_orth_cluster(T* G, int S, int r, int64_t h, int C, double tol, int* status, float* out32,
                                        __nv_bfloat16* planes, int plane_rows, size_t smem, cudaStream_t st) {
-  auto kernel = orth_cluster_kernel<BS>;
+  auto kernel = orth_cluster_kernel<BS, T>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   cudaLaunchConfig_t cfg = {};
@@ -389,19 +406,24 @@ static cudaError_t launch_orth_cluster(float* G, int S, int r, int64_t h, int C,
 }
 
 // Whether the one-launch kernel takes this shape (the slab of a CTA has to fit in shared memory).
-bool orth_cluster_fits(int r, int64_t h) {
+bool orth_cluster_fits(int r, int64_t h, size_t elem_bytes) {
   if (h > (int64_t)1 << 30) return false;
-  return cluster_size_for(r, h, 1 << 20) > 0;  // the largest admissible cluster decides
+  return cluster_size_for(r, h, 1 << 20, elem_bytes) > 0;  // the largest admissible cluster decides
 }
 
-// Cholesky-QR (one or two passes, decided on the device) of the rows of G (S x r x h fp32, in place).
-cudaError_t orth_cluster(float* G, int S, int r, int64_t h, double tol, int* status, float* out32,
-                         __nv_bfloat16* planes, int plane_rows, cudaStream_t st) {
-  const int C = cluster_size_for(r, h, S);
+// Cholesky-QR (one or two passes, decided on the device) of the rows of G (S x r x h, in place).
+template <typename T>
+cudaError_t orth_cluster(T* G, int S, int r, int64_t h, double tol, int* status, float* out32, __nv_bfloat16* planes,
+                         int plane_rows, cudaStream_t st) {
+  const int C = cluster_size_for(r, h, S, sizeof(T));
   if (C == 0) return cudaErrorInvalidValue;
   if (r >= 32)
-    return launch_orth_cluster<8>(G, S, r, h, C, tol, status, out32, planes, plane_rows, orth_geom<8>(r, h, C).total, st);
-  return launch_orth_cluster<2>(G, S, r, h, C, tol, status, out32, planes, plane_rows, orth_geom<2>(r, h, C).total, st);
+    return launch_orth_cluster<8, T>(G, S, r, h, C, tol, status, out32, planes, plane_rows,
+                                     orth_geom<8>(r, h, C, sizeof(T)).total, st);
+  return launch_orth_cluster<2, T>(G, S, r, h, C, tol, status, out32, planes, plane_rows,
+                                   orth_geom<2>(r, h, C, sizeof(T)).total, st);
 }
+template cudaError_t orth_cluster<float>(float*, int, int, int64_t, double, int*, float*, __nv_bfloat16*, int, cudaStream_t);
+template cudaError_t orth_cluster<double>(double*, int, int, int64_t, double, int*, float*, __nv_bfloat16*, int, cudaStream_t);
 
 }  // namespace dad
