@@ -448,6 +448,12 @@ def run_ours(args):
                "sample": f"{reps}x [{sample}]", "seconds": secs}
 
     if rank == 0:
+        # Conservative bound beside the streamed one: every element of A and Delta has to cross HBM at least once
+        # per layer (the passes re-read them 2*iters+1 times; nothing of a 64-256-slice launch survives in L2).
+        b_min = sum((sh.h_in + sh.h_out) * cfg.S * cfg.N * cfg.elem_bytes for sh in layers) * cfg.blocks
+        t_min_ms = b_min / (peaks["hbm_gbs"] * 1e9) * 1e3
+        compulsory = {"bytes_per_step": b_min, "t_min_ms": t_min_ms, "frac": t_min_ms / ms_per_step,
+                      "note": "t_min = bytes of A and Delta read once / measured HBM rate; the method's passes re-read them"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "bf16", "data": "synthetic",
@@ -459,7 +465,7 @@ def run_ours(args):
                            "launch": "CUDA graph replay" if args.cuda_graph else "stream launches",
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-                "kernels": kernels, "dad_full_grad": full_grad,
+                "kernels": kernels, "dad_full_grad": full_grad, "compulsory_traffic": compulsory,
                 "stream_gbs": sum(sum(v for k, v in stream_bytes_per_layer(cfg, sh, iters).items() if not k.endswith("launches"))
                                   for sh in layers) * cfg.blocks / (ms_per_step * 1e-3) / 1e9}
         print(json.dumps(line))
