@@ -150,6 +150,22 @@ dad_status dad_rank_compress_gram(const dad_layer* layer, const void* A, const v
                                   void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The same compression with the components found one after the other, the order in which Algorithm 2 is printed
+ * (Sec. 3.3.1): for j = 0 .. r-1, g <- Q0[j] made orthogonal to the components found so far and normalised;
+ * iters times  g <- M g - sum_{l<j} sigma_l^2 g_l (g_l . g)  (M = gradW^T gradW applied through D and A, Eq.
+ * "reduced_iter"; the subtraction is Eq. "peel"), orthogonalised against the found components again and
+ * normalised; then Q[j] = g, P[j] = A^T (D g), sigma_j = ||P[j]||.  A component whose remainder falls to 1e-12 of
+ * its length before the projection is set to zero.  It spans the same subspace as dad_rank_compress once both
+ * have converged, and costs r times the passes over A and D: provided to compare the two orders, not for speed.
+ * Arguments, layouts and errors as dad_rank_compress; both dtypes; products accumulate in fp64.
+ *   ws >= dad_rank_compress_sequential_workspace_bytes(layer, r, iters)
+ */
+size_t dad_rank_compress_sequential_workspace_bytes(const dad_layer* layer, int r, int iters);
+dad_status dad_rank_compress_sequential(const dad_layer* layer, const void* A, const void* D, int r, int iters,
+                                        const float* Q0, float* P, float* Q, float* sigma,
+                                        void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Gather at the aggregator (Algorithm 1, the two vertcat lines): site s's factors become rows
  * s*r .. s*r+r-1 of the stacks, and each site is charged what it sent.
  *   P, Q       DEVICE, S x r x h_in and S x r x h_out fp32 (as written by dad_rank_compress)

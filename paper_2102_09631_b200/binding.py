@@ -27,7 +27,7 @@ EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_b
            "dad_reconstruct_batched_workspace_bytes", "dad_reconstruct_batched",
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
-           "dad_rank_compress_gram",
+           "dad_rank_compress_gram", "dad_rank_compress_sequential_workspace_bytes", "dad_rank_compress_sequential",
            "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
@@ -101,6 +101,11 @@ def lib() -> ctypes.CDLL:
         L.dad_rank_compress_gram_workspace_bytes.restype = ctypes.c_size_t
         L.dad_rank_compress_gram.argtypes = [lp, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.dad_rank_compress_gram.restype = ctypes.c_int
+        L.dad_rank_compress_sequential_workspace_bytes.argtypes = [lp, ctypes.c_int, ctypes.c_int]
+        L.dad_rank_compress_sequential_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_rank_compress_sequential.argtypes = [lp, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp,
+                                                   ctypes.c_size_t, vp]
+        L.dad_rank_compress_sequential.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -278,6 +283,17 @@ def dad_rank_compress_gram(layer: dad_layer, A, D, r: int, iters: int, Q0, P, Q,
     st = lib().dad_rank_compress_gram(ctypes.byref(layer), _ptr(A), _ptr(D), r, iters, _ptr(Q0), _ptr(P), _ptr(Q),
                                       _ptr(sigma), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     _check(st, "dad_rank_compress_gram")
+
+
+def dad_rank_compress_sequential_workspace_bytes(layer: dad_layer, r: int, iters: int) -> int:
+    return int(lib().dad_rank_compress_sequential_workspace_bytes(ctypes.byref(layer), r, iters))
+
+
+def dad_rank_compress_sequential(layer: dad_layer, A, D, r: int, iters: int, Q0, P, Q, sigma, ws, stream=None):
+    """dad_rank_compress with the components found one after the other (Algorithm 2 in its printed order)."""
+    st = lib().dad_rank_compress_sequential(ctypes.byref(layer), _ptr(A), _ptr(D), r, iters, _ptr(Q0), _ptr(P), _ptr(Q),
+                                            _ptr(sigma), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_rank_compress_sequential")
 
 
 def dad_check(ws, stream=None):

@@ -184,3 +184,32 @@ def test_gram_form_refuses_what_it_does_not_take(B):
     Lb = B.make_layer(A[:, :64].bfloat16(), D[:, :64].bfloat16())
     with pytest.raises(B.DadError, match="DTYPE"):
         B.dad_rank_compress_gram(Lb, A, D, 4, 1, buf, buf, buf, None, ws)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("S,N,h_in,h_out,r,iters,dtype,raw", [
+    (3, 40, 96, 72, 5, 3, torch.float32, True),
+    (2, 300, 256, 512, 6, 2, torch.bfloat16, True),     # bf16 inputs through the general kernels, fp64 accumulation
+    (2, 5, 48, 40, 8, 2, torch.float32, False),         # batch smaller than r: components beyond the rank carry nothing
+])
+def test_sequential_form_matches_the_oracles_algorithm_2(oracle, B, S, N, h_in, h_out, r, iters, dtype, raw):
+    """dad_rank_compress_sequential (components one after the other, peel term, Sec. 3.3.1) against the oracle's
+    vector-at-a-time Algorithm 2 on every site: projected gradient, and -- where the spectrum separates the
+    components -- the vectors themselves, which the common start block fixes including their signs."""
+    dev = torch.device("cuda:0")
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 700 + N, dtype, modes=8)
+    Q0 = wl.start_block(S, r, h_out, 700 + N)
+    Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
+    L = B.make_layer(Ad, Dd)
+    P, Q, sg = (torch.empty(S, r, h_in, device=dev), torch.empty(S, r, h_out, device=dev), torch.empty(S, r, device=dev))
+    ws = B.new_workspace(B.dad_rank_compress_sequential_workspace_bytes(L, r, iters), dev)
+    B.dad_rank_compress_sequential(L, Ad, Dd, r, iters, Q0d, P, Q, sg, ws)
+    B.dad_check(ws)
+    Pn, Qn, sn = P.double().cpu().numpy(), Q.double().cpu().numpy(), sg.double().cpu().numpy()
+    for s in range(S):
+        Po, Qo, so = oracle.spi_paper(A[s], D[s], Q0[s], iters)
+        assert rel(Pn[s].T @ Qn[s], Po.T @ Qo) <= 1e-5
+        if raw:
+            assert rel(Qn[s], Qo) <= 1e-4 and rel(Pn[s], Po) <= 1e-4
+            assert np.abs(sn[s] - so).max() <= 1e-5 * so.max()
+            assert np.linalg.norm(Qn[s] @ Qn[s].T - np.eye(r)) <= 1e-5
