@@ -122,6 +122,7 @@ def test_config3_encoder_layer_projections(oracle, B):
     (257, 200, 136, 10, 2, torch.bfloat16),           # widths that are multiples of 8 but of no tile
     (100, 70, 50, 7, 2, torch.bfloat16),              # widths that are not multiples of 8: general kernels
     (130, 96, 40, 5, 3, torch.float32),
+    (2048, 512, 256, 8, 2, torch.float32),            # recurrent layer 512 -> 256 over batch x time rows, fp32
     (72, 264, 2048, 48, 2, torch.float32),            # fp64 vectors, slab of the one-launch Cholesky-QR still fits
     (72, 264, 4096, 64, 1, torch.float32),            # fp64 vectors too wide for it: the multi-kernel Cholesky-QR
 ])
