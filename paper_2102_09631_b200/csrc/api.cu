@@ -218,7 +218,11 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
     DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, nullptr, nullptr, Fz, hi, part, ctr_cols, status, st));     // Z = Y^T A
     DAD_STEP(umma_rows_dot(tmA_rows, tmFz, S, N, hi, r, Yt, w.Npad, status, st));                                  // W = A Z^T
     DAD_STEP(umma_cols_acc(tmD_cols, tmYt, S, N, ho, r, Q, nullptr, nullptr, 0, part, ctr_cols, status, st));       // Gt = W^T D
-    if (orth_cluster_fits(r, ho)) {
+    if (orth_split_preferred(r, ho, S)) {
+      DAD_STEP(orth_split(Q, S, r, ho, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, nullptr, Fq, rp, st));
+    } else if (orth_mma_fits(r, ho)) {
+      DAD_STEP(orth_mma(Q, S, r, ho, tol, status, nullptr, Fq, rp, st));
+    } else if (orth_cluster_fits(r, ho)) {
       DAD_STEP(orth_cluster(Q, S, r, ho, tol, status, nullptr, Fq, rp, st));
     } else {
       DAD_STEP(cholqr_pass<float>(Q, S, r, ho, 0, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status,

@@ -107,6 +107,16 @@ bool orth_cluster_fits(int r, int64_t h, size_t elem_bytes = 4);
 template <typename T>
 cudaError_t orth_cluster(T* G, int S, int r, int64_t h, double tol, int* status, float* out32,
                          __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
+// fp32 storage with the Gram and substitution phases on the fp64 matrix-multiply unit (orth_mma.cu).
+bool orth_mma_fits(int r, int64_t h);
+cudaError_t orth_mma(float* G, int S, int r, int64_t h, double tol, int* status, float* out32, __nv_bfloat16* planes,
+                     int plane_rows, cudaStream_t st);
+// The same phases as two launches per pass, the factorisation once per site; preferred for many sites at r >= 32.
+// Scratch as for cholqr_pass (gram_partial, gram, tratio, dead, need2, counters), which is large enough when preferred.
+bool orth_split_preferred(int r, int64_t h, int S);
+cudaError_t orth_split(float* G, int S, int r, int64_t h, double tol, double* gram_partial, double* gram, double* tratio,
+                       unsigned char* dead, int* need2, unsigned* counters, int* status, float* out32,
+                       __nv_bfloat16* planes, int plane_rows, cudaStream_t st);
 
 // C[a][b] = sum_{s,n} X[s][n][a] * Y[s][n][b]  (fp32 FMA), C: hx x hy fp32 contiguous
 cudaError_t gemm_tn_simt(dad_dtype dt, const void* X, int64_t ldX, int64_t strideX, const void* Y,

@@ -121,6 +121,12 @@ def test_config3_encoder_layer_projections(oracle, B):
     (515, 4096, 1024, 64, 1, torch.bfloat16),         # ffn_down at the largest rank, odd row count
     (257, 200, 136, 10, 2, torch.bfloat16),           # widths that are multiples of 8 but of no tile
     (100, 70, 50, 7, 2, torch.bfloat16),              # widths that are not multiples of 8: general kernels
+    (200, 256, 520, 24, 2, torch.bfloat16),           # ranks that pad to 3, 4, 5, 6, 7 row blocks of eight in the
+    (200, 256, 512, 32, 2, torch.bfloat16),           # orthonormalisation (odd counts leave a middle block unpaired),
+    (200, 512, 1024, 40, 2, torch.bfloat16),          # slabs of one to eight CTAs per site
+    (200, 384, 776, 48, 1, torch.bfloat16),
+    (200, 384, 768, 56, 1, torch.bfloat16),
+    (260, 256, 4096, 64, 2, torch.bfloat16),          # widest slab at the largest rank, two iterations
     (130, 96, 40, 5, 3, torch.float32),
     (2048, 512, 256, 8, 2, torch.float32),            # recurrent layer 512 -> 256 over batch x time rows, fp32
     (72, 264, 2048, 48, 2, torch.float32),            # fp64 vectors, slab of the one-launch Cholesky-QR still fits
