@@ -350,6 +350,26 @@ def run_ours(args):
             roofline = {"bound": "hbm", "kernel": name, "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": None, "traffic": None, "peak_source": peaks["source"]}
 
+    # ---- the reconstruction products (P^T Q over the S r stacked rows) of the step, from the same event pass ----
+    reconstruct = None
+    rec = kernels.get("gemm_tn_tc") or kernels.get("gemm_tn_simt")
+    if rec:
+        K = cfg.S * r
+        bf16 = "gemm_tn_tc" in kernels
+        terms = 3 if bf16 else 1           # bf16 math multiplies two-term splits of the fp32 factors: three products
+        flops = sum(2.0 * K * sh.h_in * sh.h_out for sh in layers) * cfg.blocks
+        out_bytes = sum(4.0 * sh.h_in * sh.h_out for sh in layers) * cfg.blocks
+        in_bytes = sum((2.0 * terms if bf16 else 4.0) * K * (sh.h_in + sh.h_out) for sh in layers) * cfg.blocks
+        t = rec["ms_per_step"] * 1e-3
+        tf_exec = terms * flops / t / 1e12
+        reconstruct = {"kernel": "gemm_tn_tc" if bf16 else "gemm_tn_simt", "contraction": K, "products": terms,
+                       "ms_per_step": rec["ms_per_step"], "tflops_algorithmic": flops / t / 1e12,
+                       "tflops_executed": tf_exec,
+                       "frac_tensor_executed": tf_exec / peaks["bf16_tflops"] if bf16 else None,
+                       "gbs": (out_bytes + in_bytes) / t / 1e9, "frac_hbm": (out_bytes + in_bytes) / t / 1e9 / peaks["hbm_gbs"],
+                       "bound": "tensor" if bf16 and terms * flops / (peaks["bf16_tflops"] * 1e12) >
+                                (out_bytes + in_bytes) / (peaks["hbm_gbs"] * 1e9) else "hbm"}
+
     # ---- the uncompressed dAD gradient (sum_s A_s^T D_s) of each layer shape: the tensor-bound product ----
     full_grad = None
     if not args.no_full_grad:
@@ -465,7 +485,7 @@ def run_ours(args):
                            "launch": "CUDA graph replay" if args.cuda_graph else "stream launches",
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-                "kernels": kernels, "dad_full_grad": full_grad, "compulsory_traffic": compulsory,
+                "kernels": kernels, "reconstruct": reconstruct, "dad_full_grad": full_grad, "compulsory_traffic": compulsory,
                 "stream_gbs": sum(sum(v for k, v in stream_bytes_per_layer(cfg, sh, iters).items() if not k.endswith("launches"))
                                   for sh in layers) * cfg.blocks / (ms_per_step * 1e-3) / 1e9}
         print(json.dumps(line))

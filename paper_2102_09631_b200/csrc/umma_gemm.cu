@@ -698,7 +698,14 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
                (int)hy, C);
     return err;
   }
-  if (g.bn == 256) return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+  // Short contractions (the reconstruction: 3 S r rows) spend as long in the epilogue -- 128 KB of fp32 per tile -- as in
+  // the MMAs: two shallow CTAs per SM, one draining its accumulator while the other multiplies, instead of one deep one.
+  const bool shallow = p.kb_per_split <= 64;
+  if (g.bn == 256) {
+    if (shallow) return launch_umma<256, true, true, 1, EPI_C, 2>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+    return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+  }
+  if (shallow) return launch_umma<128, true, true, 1, EPI_C, 3>(tmX, tmY, p, grid, "gemm_tn_tc", st);
   return launch_umma<128, true, true, 1, EPI_C, 6>(tmX, tmY, p, grid, "gemm_tn_tc", st);
 }
 
