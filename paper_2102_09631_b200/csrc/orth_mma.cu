@@ -23,12 +23,14 @@
 //     every CTA, so all CTAs factor the identical matrix and take identical decisions.  Vectors cross
 //     HBM once each way.  Every CTA repeats the factorisation, which is a latency chain: right for few
 //     sites.
-//   * two launches per pass for many sites at large r: (1) partial Gram per 128-column chunk, the last
+//   * two launches per pass for many sites at large r: (1) partial Gram per 256-column chunk, the last
 //     CTA of a site to arrive adds the partials in chunk order, factors and stores the M matrices;
 //     (2) every chunk applies them.  The factorisation runs once per site and under other sites' Gram
 //     work.
 // All sums run in a fixed order: two runs give identical bits.
 #include <cooperative_groups.h>
+
+#include <algorithm>
 
 #include "common.cuh"
 
@@ -42,7 +44,8 @@ constexpr double kSecondPassBelowSq = 1e-10;  // (1e-5)^2: one fp64 pass leaves 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr size_t kSmemLimit = 200 * 1024;
-constexpr int kSplitW = 128;  // columns per CTA of the two-launch arrangement
+constexpr int kFactorW = 256;  // columns per CTA of the two-launch arrangement: Gram + factorisation kernel
+constexpr int kApplyW = 128;   // ... and substitution kernel
 
 struct MmaGeom {
   int rp, nb, nt;  // padded rank, row blocks of 8, tiles of the lower triangle
@@ -577,16 +580,15 @@ orth_mma_kernel(float* __restrict__ G, int r, int64_t h, int C, int W, double to
 // =====================================================================================================================
 template <int NB>
 __global__ void __launch_bounds__(kThreads, 2)
-orth_split_factor_kernel(const float* __restrict__ G, int r, int64_t h, int chunks, int pass, double tol,
+orth_split_factor_kernel(const float* __restrict__ G, int S, int r, int64_t h, int chunks, int pass, double tol,
                          double* __restrict__ partial, double* __restrict__ Mt, double* __restrict__ ratio1,
                          unsigned char* __restrict__ dead, int* __restrict__ need2, unsigned* __restrict__ counters,
                          int* __restrict__ status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int rp = NB * 8, nt = NB * (NB + 1) / 2;
-  const int s = blockIdx.y, chunk = blockIdx.x;
+  const int chunk = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (pass == 1 && need2[s] == 0) return;
-  const MmaGeom geo = mma_geom(r, kSplitW);
+  const MmaGeom geo = mma_geom(r, kFactorW);
   // the factorisation (last CTA only) reuses the slab's place for L: the slab is spent by then
   float* slab = reinterpret_cast<float*>(smem_raw);
   double* Lm = reinterpret_cast<double*>(smem_raw);
@@ -601,11 +603,16 @@ orth_split_factor_kernel(const float* __restrict__ G, int r, int64_t h, int chun
   const FactorState f = factor_state(vec, rp, dead_row, &need2_s);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int Wp = geo.Wp, LR = geo.LR;
-
-  load_slab(slab, G + (int64_t)s * r * h, r, rp, h, (int64_t)chunk * kSplitW, kSplitW, Wp, tid);
   fill_tile_table(tile_bi, tile_bj, nt, tid);
+
+  // First pass: one site per CTA row.  Second pass: a small grid walks over the sites and skips those that do not
+  // need it (nearly always all of them), so the launch costs next to nothing.
+  for (int s = blockIdx.y; s < S; s += gridDim.y) {
+  if (pass == 1 && need2[s] == 0) continue;
+  __syncthreads();  // the previous site's shared memory is no longer in use
+  load_slab(slab, G + (int64_t)s * r * h, r, rp, h, (int64_t)chunk * kFactorW, kFactorW, Wp, tid);
   __syncthreads();
-  gram_tiles<NB>(slab, kSplitW, Wp, tiles, warp, lane);
+  gram_tiles<NB>(slab, kFactorW, Wp, tiles, warp, lane);
   double* mine = partial + ((size_t)s * chunks + chunk) * nt * 64;
   for (int e = tid; e < nt * 64; e += kThreads) mine[e] = tiles[e];
   __threadfence();
@@ -616,7 +623,7 @@ orth_split_factor_kernel(const float* __restrict__ G, int r, int64_t h, int chun
     if (is_last) counters[s] = 0u;
   }
   __syncthreads();
-  if (!is_last) return;
+  if (!is_last) continue;
   __threadfence();
 
   // ---- sum the chunk partials in chunk order (loads issued eight at a time) into L ----
@@ -661,31 +668,35 @@ orth_split_factor_kernel(const float* __restrict__ G, int r, int64_t h, int chun
     dead[(size_t)s * r + tid] = f.dead_row[tid];
   }
   if (tid == 0 && pass == 0) need2[s] = need2_s;
+  }
 }
 
 template <int NB>
 __global__ void __launch_bounds__(kThreads, 3)
-orth_split_apply_kernel(float* __restrict__ G, int r, int64_t h, int pass, const double* __restrict__ Mt,
+orth_split_apply_kernel(float* __restrict__ G, int S, int r, int64_t h, int pass, const double* __restrict__ Mt,
                         const int* __restrict__ need2, float* __restrict__ out32, __nv_bfloat16* __restrict__ planes,
                         int plane_rows) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int rp = NB * 8, nt = NB * (NB + 1) / 2;
-  const int s = blockIdx.y, chunk = blockIdx.x;
+  const int chunk = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (pass == 1 && need2[s] == 0) return;
-  const MmaGeom geo = mma_geom(r, kSplitW);
+  const MmaGeom geo = mma_geom(r, kApplyW);
   float* slab = reinterpret_cast<float*>(smem_raw);
   double* tiles = reinterpret_cast<double*>(smem_raw + geo.off_tiles);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t c0 = (int64_t)chunk * kApplyW;
+  for (int s = blockIdx.y; s < S; s += gridDim.y) {  // second pass: a small grid walks over the sites
+  if (pass == 1 && need2[s] == 0) continue;
+  __syncthreads();
   float* Gs = G + (int64_t)s * r * h;
-  const int64_t c0 = (int64_t)chunk * kSplitW;
   const double* Ms = Mt + (size_t)s * nt * 64;
   for (int e = tid; e < nt * 64; e += kThreads) tiles[e] = Ms[e];
-  load_slab(slab, Gs, r, rp, h, c0, kSplitW, geo.Wp, tid);
+  load_slab(slab, Gs, r, rp, h, c0, kApplyW, geo.Wp, tid);
   __syncthreads();
-  solve_slab(slab, tiles, NB, kSplitW, geo.Wp, warp, lane);
+  solve_slab(slab, tiles, NB, kApplyW, geo.Wp, warp, lane);
   __syncthreads();
-  store_slab(slab, Gs, s, r, h, c0, kSplitW, geo.Wp, out32, planes, plane_rows, tid);
+  store_slab(slab, Gs, s, r, h, c0, kApplyW, geo.Wp, out32, planes, plane_rows, tid);
+  }
 }
 
 template <int NB>
@@ -718,23 +729,25 @@ template <int NB>
 static cudaError_t launch_orth_split(float* G, int S, int r, int64_t h, double tol, double* partial, double* Mt,
                                      double* ratio1, unsigned char* dead, int* need2, unsigned* counters, int* status,
                                      float* out32, __nv_bfloat16* planes, int plane_rows, cudaStream_t st) {
-  const MmaGeom geo = mma_geom(r, kSplitW);
-  const int chunks = (int)ceil_div(h, kSplitW);
+  const MmaGeom geo = mma_geom(r, kFactorW), geo_a = mma_geom(r, kApplyW);
+  const int chunks = (int)ceil_div(h, kFactorW), chunks_a = (int)ceil_div(h, kApplyW);
   const size_t lbytes = sizeof(double) * (size_t)geo.rp * geo.LR;
   const size_t smem_f =
       (lbytes > geo.off_tiles ? lbytes : geo.off_tiles) + sizeof(double) * (64 * (size_t)geo.nt + 5 * (size_t)geo.rp);
-  const size_t smem_a = geo.off_tiles + sizeof(double) * 64 * (size_t)geo.nt;
+  const size_t smem_a = geo_a.off_tiles + sizeof(double) * 64 * (size_t)geo_a.nt;
   cudaError_t err =
       cudaFuncSetAttribute(orth_split_factor_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f);
   if (err != cudaSuccess) return err;
   err = cudaFuncSetAttribute(orth_split_apply_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_a);
   if (err != cudaSuccess) return err;
-  const dim3 grid((unsigned)chunks, (unsigned)S);
   for (int pass = 0; pass < 2; ++pass) {
-    DAD_LAUNCH(err, "orth_split_factor", (orth_split_factor_kernel<NB>), grid, kThreads, smem_f, st, G, r, h, chunks, pass,
-               tol, partial, Mt, ratio1, dead, need2, counters, status);
-    DAD_LAUNCH(err, "orth_split_apply", (orth_split_apply_kernel<NB>), grid, kThreads, smem_a, st, G, r, h, pass, Mt, need2,
-               out32, planes, plane_rows);
+    // second pass: about two CTAs per SM in all, each walking over the sites
+    const int rows_f = pass == 0 ? S : (int)std::max<int64_t>(1, std::min<int64_t>(S, 2 * 148 / chunks));
+    const int rows_a = pass == 0 ? S : (int)std::max<int64_t>(1, std::min<int64_t>(S, 2 * 148 / chunks_a));
+    DAD_LAUNCH(err, "orth_split_factor", (orth_split_factor_kernel<NB>), dim3((unsigned)chunks, (unsigned)rows_f), kThreads,
+               smem_f, st, G, S, r, h, chunks, pass, tol, partial, Mt, ratio1, dead, need2, counters, status);
+    DAD_LAUNCH(err, "orth_split_apply", (orth_split_apply_kernel<NB>), dim3((unsigned)chunks_a, (unsigned)rows_a), kThreads,
+               smem_a, st, G, S, r, h, pass, Mt, need2, out32, planes, plane_rows);
   }
   return err;
 }
@@ -750,7 +763,7 @@ bool orth_mma_fits(int r, int64_t h) {
 // are sized for the multi-kernel Cholesky-QR (S x ceil(h / 64) x r x r doubles of partials, S x r x r of factor).
 bool orth_split_preferred(int r, int64_t h, int S) {
   if (r < 32 || r > DAD_MAX_RANK) return false;
-  const MmaGeom geo = mma_geom(r, kSplitW);
+  const MmaGeom geo = mma_geom(r, kFactorW);
   if ((size_t)geo.nt * 64 > (size_t)r * r) return false;
   const int C = mma_cluster_size(r, h, S);
   return C == 0 || (int64_t)S * C > 2 * 148;

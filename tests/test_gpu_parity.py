@@ -207,6 +207,24 @@ def test_rank_exceeding_true_rank_is_exact(oracle, B):
         assert np.all(g["sigma"][s][N:] == 0.0)
 
 
+@pytest.mark.parametrize("iters,dependent_start", [(2, False), (1, True)])
+def test_many_sites_at_large_rank(oracle, B, iters, dependent_start):
+    """160 sites at r = 32: more CTAs than the GPU holds at once, so the orthonormalisation takes its two-launch
+    form (Gram + one factorisation per site, then the substitution).  With two start vectors that repeat others
+    (one of them scaled) the iterate has two exactly dependent vectors: their pivots reach the floor, the second
+    pass runs, and those two come out as zeros -- in the oracle too, so the live sets must agree."""
+    S, N, h_in, h_out, r = 160, 72, 128, 256, 32
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 587, torch.bfloat16)
+    Q0 = wl.start_block(S, r, h_out, 587)
+    if dependent_start:
+        Q0[:, r - 1] = Q0[:, 0]
+        Q0[:, 9] = 2.0 * Q0[:, 4]
+    g, o = check_layer(oracle, B, A, D, Q0, r, iters, TOL[torch.bfloat16], ortho_tol=1e-3)
+    if dependent_start:
+        for s in (0, 77, S - 1):
+            assert [j for j in range(r) if np.all(g["Q"][s][j] == 0.0)] == [9, r - 1]
+
+
 def test_edge_shapes(oracle, B):
     # one row, one site, r = 1; r = min(h); zero iterations; strided (non-contiguous) rows and sites
     A, D = wl.gaussian_layer(1, 1, 8, 8, 1)
