@@ -355,7 +355,11 @@ __device__ __forceinline__ void cholesky_panels(double* __restrict__ Lm, int LR,
         const bool usable = !bad && orig[jj] > 0.0;
         const double d = D[jj][jj];
         const double il_raw = rsqrt(d);  // started at once; the decisions below run beside it
-        const bool ok = d > floor_[jj];  // a pivot at or below the floor (or not a number) is raised to it
+        // A pivot at or below the floor is raised to it.  Both are compared as integers (same order as the values for
+        // a positive floor; a negative pivot has the sign bit set and is smaller): the fp64 comparison would take
+        // longer than the reciprocal square root beside it and hold up the choice between the two candidates.
+        // (A floor that is not positive or not a number belongs to an unusable vector, which is zeroed whatever ok is.)
+        const bool ok = __double_as_longlong(d) > __double_as_longlong(floor_[jj]);
         const double piv = ok ? d : floor_[jj];
         // zeroing rule: first pass never (known ahead, so the choice of the scale below waits for the floor test
         // only); second pass: total remainder (R1_jj R2_jj)^2 against tol^2 of the squared length before the first
