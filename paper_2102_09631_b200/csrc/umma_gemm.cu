@@ -607,7 +607,13 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
   p.status = status;
   dim3 grid((unsigned)ceil_div(h, 128), (unsigned)p.splits, (unsigned)S);
   switch (umma_rank_pad(r)) {
-    case 16: return launch_umma<16, true, false, 2, EPI_Z, 5>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+    // r <= 16: when the launch has CTAs for many waves, five shallow CTAs per SM stream better than two deep ones, as
+    // in rows_dot (2 / 3 / 4 / 5 stages: 30.8 / 31.0 / 31.2 / 31.5 ms per benchmark step of 2048-CTA launches); with
+    // fewer CTAs the 740 slots of the shallow form leave a nearly empty last wave (768 CTAs: 9.2 -> 10.7 ms).
+    case 16:
+      if ((int64_t)grid.x * grid.y * grid.z >= 12 * 148)
+        return launch_umma<16, true, false, 2, EPI_Z, 2>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+      return launch_umma<16, true, false, 2, EPI_Z, 5>(tmX, tmYt, p, grid, "cols_acc_tc", st);
     case 32: return launch_umma<32, true, false, 2, EPI_Z, 4>(tmX, tmYt, p, grid, "cols_acc_tc", st);
     default: return launch_umma<64, true, false, 2, EPI_Z, 3>(tmX, tmYt, p, grid, "cols_acc_tc", st);
   }
