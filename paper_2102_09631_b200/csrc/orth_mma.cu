@@ -75,15 +75,17 @@ __host__ __device__ inline MmaGeom mma_geom(int r, int W) {
 
 inline int columns_per_cta(int64_t h, int C) { return (int)((ceil_div(h, C) + 7) / 8 * 8); }
 
-// CTAs per site of the one-launch arrangement: as few as still give every SM two CTAs (each CTA of a cluster
-// repeats the r x r factorisation), more if the slab would not fit otherwise; no slabs narrower than 128 columns.
+// CTAs per site of the one-launch arrangement: as few as still give every SM a CTA (each CTA of a cluster repeats the
+// r x r factorisation, and a launch that fits the GPU in one wave beats a finer one in two: 256 sites at r = 16,
+// h = 1024 take 25 us as 256 CTAs, 36 us as 512), more if the slab would not fit otherwise; no slabs narrower than
+// 128 columns.
 inline int mma_cluster_size(int r, int64_t h, int S) {
   int best = 0;
   for (int C = 1; C <= 8; C *= 2) {
     if (C > 1 && h / C < 128) break;
     if (mma_geom(r, columns_per_cta(h, C)).total > kSmemLimit) continue;
     best = C;
-    if ((int64_t)S * C >= 2 * 148) break;
+    if ((int64_t)S * C >= 148) break;
   }
   return best;
 }
