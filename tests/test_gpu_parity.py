@@ -209,11 +209,11 @@ def test_rank_exceeding_true_rank_is_exact(oracle, B):
 
 @pytest.mark.parametrize("iters,dependent_start", [(2, False), (1, True)])
 def test_many_sites_at_large_rank(oracle, B, iters, dependent_start):
-    """160 sites at r = 32: more CTAs than the GPU holds at once, so the orthonormalisation takes its two-launch
+    """320 sites at r = 32: more CTAs than the GPU holds at once, so the orthonormalisation takes its two-launch
     form (Gram + one factorisation per site, then the substitution).  With two start vectors that repeat others
     (one of them scaled) the iterate has two exactly dependent vectors: their pivots reach the floor, the second
     pass runs, and those two come out as zeros -- in the oracle too, so the live sets must agree."""
-    S, N, h_in, h_out, r = 160, 72, 128, 256, 32
+    S, N, h_in, h_out, r = 320, 72, 128, 256, 32
     A, D = wl.gaussian_layer(S, N, h_in, h_out, 587, torch.bfloat16)
     Q0 = wl.start_block(S, r, h_out, 587)
     if dependent_start:
