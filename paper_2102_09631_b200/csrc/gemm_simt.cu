@@ -95,13 +95,36 @@ __global__ void copy_two_kernel(const float* __restrict__ a, float* __restrict__
   }
 }
 
+// The same with 16-byte accesses: na and nb count float4 elements.
+__global__ void copy_two_vec_kernel(const float4* __restrict__ a, float4* __restrict__ a_out, size_t na,
+                                    const float4* __restrict__ b, float4* __restrict__ b_out, size_t nb) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < na + nb; i += stride) {
+    if (i < na) {
+      if (a_out != a) a_out[i] = a[i];
+    } else {
+      if (b_out != b) b_out[i - na] = b[i - na];
+    }
+  }
+}
+
 cudaError_t copy_two(const float* a, float* a_out, size_t na, const float* b, float* b_out, size_t nb,
                      cudaStream_t st) {
   cudaError_t err = cudaSuccess;
-  size_t blocks = (na + nb + 255) / 256;
+  const bool vec = na % 4 == 0 && nb % 4 == 0 &&
+                   ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(a_out) | reinterpret_cast<uintptr_t>(b) |
+                     reinterpret_cast<uintptr_t>(b_out)) & 15) == 0;
+  const size_t items = vec ? (na + nb) / 4 : na + nb;
+  size_t blocks = (items + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  DAD_LAUNCH(err, "gather_copy", copy_two_kernel, (unsigned)blocks, 256, 0, st, a, a_out, na, b, b_out, nb);
+  if (vec) {
+    DAD_LAUNCH(err, "gather_copy", copy_two_vec_kernel, (unsigned)blocks, 256, 0, st, reinterpret_cast<const float4*>(a),
+               reinterpret_cast<float4*>(a_out), na / 4, reinterpret_cast<const float4*>(b),
+               reinterpret_cast<float4*>(b_out), nb / 4);
+  } else {
+    DAD_LAUNCH(err, "gather_copy", copy_two_kernel, (unsigned)blocks, 256, 0, st, a, a_out, na, b, b_out, nb);
+  }
   return err;
 }
 
@@ -132,14 +155,43 @@ __global__ void split_planes_kernel(const float* __restrict__ in, int r, int64_t
   }
 }
 
+// Four elements per thread (h a multiple of four, `in` 16-byte and `planes` 8-byte aligned); n counts quads.
+__global__ void split_planes_vec_kernel(const float4* __restrict__ in, int r, int64_t h4, __nv_bfloat16* __restrict__ planes,
+                                        int plane_rows, size_t n) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const size_t c = i % (size_t)h4, sj = i / (size_t)h4;
+    const size_t j = sj % (size_t)r, s = sj / (size_t)r;
+    const float4 v = in[i];
+    const float f[4] = {v.x, v.y, v.z, v.w};
+    __align__(8) __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      hi[u] = __float2bfloat16_rn(f[u]);
+      lo[u] = __float2bfloat16_rn(f[u] - __bfloat162float(hi[u]));
+    }
+    uint2* ph = reinterpret_cast<uint2*>(planes + ((s * 2 + 0) * plane_rows + j) * (size_t)(h4 * 4)) + c;
+    uint2* pl = reinterpret_cast<uint2*>(planes + ((s * 2 + 1) * plane_rows + j) * (size_t)(h4 * 4)) + c;
+    *ph = *reinterpret_cast<const uint2*>(hi);
+    *pl = *reinterpret_cast<const uint2*>(lo);
+  }
+}
+
 cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16* planes, int plane_rows,
                          cudaStream_t st) {
   cudaError_t err = cudaSuccess;
   const size_t n = (size_t)S * r * h;
-  size_t blocks = (n + 255) / 256;
+  const bool vec = h % 4 == 0 && (reinterpret_cast<uintptr_t>(in) & 15) == 0 && (reinterpret_cast<uintptr_t>(planes) & 7) == 0;
+  const size_t items = vec ? n / 4 : n;
+  size_t blocks = (items + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  DAD_LAUNCH(err, "split_planes", split_planes_kernel, (unsigned)blocks, 256, 0, st, in, r, h, planes, plane_rows, n);
+  if (vec) {
+    DAD_LAUNCH(err, "split_planes", split_planes_vec_kernel, (unsigned)blocks, 256, 0, st,
+               reinterpret_cast<const float4*>(in), r, h / 4, planes, plane_rows, items);
+  } else {
+    DAD_LAUNCH(err, "split_planes", split_planes_kernel, (unsigned)blocks, 256, 0, st, in, r, h, planes, plane_rows, n);
+  }
   return err;
 }
 
@@ -192,11 +244,41 @@ __global__ void __launch_bounds__(256) row_norms_kernel(const T* __restrict__ M,
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
-  double acc = 0.0;
-  for (int64_t c = lane; c < h; c += 32) {
-    const double v = (double)M[row * h + c];
-    acc += v * v;
+  double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;  // four partial sums per lane: loads and additions overlap
+  const T* Mr = M + row * h;
+  int64_t c = lane;
+  if constexpr (sizeof(T) == 4) {
+    if ((h & 3) == 0 && (reinterpret_cast<uintptr_t>(M) & 15) == 0) {  // 16-byte loads, two in flight per lane
+      const float4* M4 = reinterpret_cast<const float4*>(Mr);
+      const int64_t h4 = h / 4;
+      int64_t q = lane;
+      for (; q + 32 < h4; q += 64) {
+        const float4 u = M4[q], w = M4[q + 32];
+        a0 += (double)u.x * u.x + (double)u.y * u.y;
+        a1 += (double)u.z * u.z + (double)u.w * u.w;
+        a2 += (double)w.x * w.x + (double)w.y * w.y;
+        a3 += (double)w.z * w.z + (double)w.w * w.w;
+      }
+      for (; q < h4; q += 32) {
+        const float4 u = M4[q];
+        a0 += (double)u.x * u.x + (double)u.y * u.y;
+        a1 += (double)u.z * u.z + (double)u.w * u.w;
+      }
+      c = h;  // nothing left for the scalar loops
+    }
   }
+  for (; c + 96 < h; c += 128) {
+    const double v0 = (double)Mr[c], v1 = (double)Mr[c + 32], v2 = (double)Mr[c + 64], v3 = (double)Mr[c + 96];
+    a0 += v0 * v0;
+    a1 += v1 * v1;
+    a2 += v2 * v2;
+    a3 += v3 * v3;
+  }
+  for (; c < h; c += 32) {
+    const double v = (double)Mr[c];
+    a0 += v * v;
+  }
+  double acc = (a0 + a1) + (a2 + a3);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
   if (lane == 0) out[row] = (float)sqrt(acc);
