@@ -324,6 +324,36 @@ def test_compress_at_full_size_on_sampled_sites(oracle, B):
     assert list(plan.bytes_tx) == [oracle.bytes_rank(cfg.r, shape.h_in, shape.h_out)] * cfg.S
 
 
+def test_stacked_call_at_the_benchmarks_launch_shape(oracle, B):
+    """The call the benchmark times for the attention projections of the GPT-2-medium configuration: the
+    1024 -> 1024 layers of four consecutive blocks stacked as 16 x 16 = 256 slices of one call (r = 16, three
+    iterations), i.e. 2048-CTA launches of both thin products, the one-wave Cholesky-QR and the batched
+    reconstruction.  The oracle recomputes three sampled sites and, for one whole layer of the stack, the
+    reconstructed gradient from the same inputs."""
+    dev = torch.device("cuda:0")
+    cfg = wl.CONFIGS[5]
+    S, groups, r, iters = cfg.S, 16, cfg.r, cfg.iters
+    shape = cfg.layers[0]
+    assert (shape.h_in, shape.h_out) == (1024, 1024)
+    A, D = wl.decaying_layer(S * groups, cfg.N, shape.h_in, shape.h_out, 9051, torch.bfloat16, device=dev)
+    Q0 = wl.start_block(S * groups, r, shape.h_out, 9051, dev)
+    plan = B.LayerPlan(A, D, r, iters, groups=groups)
+    grads = plan.step(A, D, Q0)
+    B.dad_check(plan.ws)
+    sites = [0, 101, S * groups - 1]
+    Po, Qo, _ = oracle.spi_block(A[sites].cpu(), D[sites].cpu(), Q0[sites].cpu(), iters)
+    for i, s in enumerate(sites):
+        got = plan.P[s].double().cpu().numpy().T @ plan.Q[s].double().cpu().numpy()
+        assert rel(got, Po[i].T @ Qo[i]) <= 2e-2
+        Qg = plan.Q[s].double().cpu().numpy()
+        assert np.linalg.norm(Qg @ Qg.T - np.eye(r)) <= 1e-3
+    g = 6                                   # one whole layer of the stack: its 16 sites and its gradient
+    sl = slice(g * S, (g + 1) * S)
+    o = oracle.rank_dad_layer(A[sl].cpu(), D[sl].cpu(), Q0[sl].cpu(), iters)
+    assert rel(grads[g].double().cpu().numpy(), o["grad"]) <= 2e-2
+    assert list(plan.bytes_tx)[sl] == [int(x) for x in o["bytes_tx"]]
+
+
 def test_stacked_layers_match_separate_calls(oracle, B):
     """Several layers of one shape stacked as extra slices of one call (groups > 1) give, layer by layer,
     what separate calls give (up to the order of the split sums) and agree with the oracle."""
