@@ -324,15 +324,16 @@ def test_compress_at_full_size_on_sampled_sites(oracle, B):
     assert list(plan.bytes_tx) == [oracle.bytes_rank(cfg.r, shape.h_in, shape.h_out)] * cfg.S
 
 
-def test_stacked_call_at_the_benchmarks_launch_shape(oracle, B):
+@pytest.mark.parametrize("r,iters", [(16, 3), (64, 1)])
+def test_stacked_call_at_the_benchmarks_launch_shape(oracle, B, r, iters):
     """The call the benchmark times for the attention projections of the GPT-2-medium configuration: the
-    1024 -> 1024 layers of four consecutive blocks stacked as 16 x 16 = 256 slices of one call (r = 16, three
-    iterations), i.e. 2048-CTA launches of both thin products, the one-wave Cholesky-QR and the batched
-    reconstruction.  The oracle recomputes three sampled sites and, for one whole layer of the stack, the
-    reconstructed gradient from the same inputs."""
+    1024 -> 1024 layers of four consecutive blocks stacked as 16 x 16 = 256 slices of one call, i.e. 2048-CTA
+    launches of both thin products and the batched reconstruction; at r = 16 (three iterations) the one-wave
+    Cholesky-QR, at r = 64 (the sweep's largest rank) its two-launch form over 256 sites.  The oracle recomputes
+    three sampled sites and, for one whole layer of the stack, the reconstructed gradient from the same inputs."""
     dev = torch.device("cuda:0")
     cfg = wl.CONFIGS[5]
-    S, groups, r, iters = cfg.S, 16, cfg.r, cfg.iters
+    S, groups = cfg.S, 16
     shape = cfg.layers[0]
     assert (shape.h_in, shape.h_out) == (1024, 1024)
     A, D = wl.decaying_layer(S * groups, cfg.N, shape.h_in, shape.h_out, 9051, torch.bfloat16, device=dev)
