@@ -103,7 +103,8 @@ GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_ope
   w.counters = off;
   off = align_up(off + tiles * sizeof(unsigned), 256);
   w.partial = off;
-  off = align_up(off + (g.splits > 1 ? tiles * (size_t)g.splits * (size_t)g.bm * (size_t)g.bn * 4 : 0), 256);
+  const size_t slots = (size_t)g.splits + (g.rem_ctas > 0 ? 1 : 0);  // partial tiles per output tile
+  off = align_up(off + (slots > 1 ? tiles * slots * (size_t)g.bm * (size_t)g.bn * 4 : 0), 256);
   w.Xb = w.Yb = off;
   if (convert_operands) {
     w.Xb = off;

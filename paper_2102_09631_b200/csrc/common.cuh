@@ -145,7 +145,9 @@ int umma_cols_acc_splits(int S, int64_t N, int64_t h);
 // bk contraction rows (the row count of the operands' TMA boxes), `splits` CTAs share a tile's contraction.
 struct GemmPlan {
   int bm, bn, bk, splits, batch;
+  int rem_ctas;                          // 256 x 256 tiles: CTAs that take the tail of every tile's contraction
   int64_t tiles, k_blocks, kb_per_site;  // tiles: per batch entry
+  int64_t kb_per_split;                  // blocks of each of the `splits` equal parts
 };
 // batch > 1: that many independent products of one site each (S must be 1) in one launch.
 GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch);

@@ -41,6 +41,8 @@ struct UmmaParams {
   int kb_per_split;
   int splits;
   int kb_per_site;   // gemm_tn over sites: blocks per site (site = block / kb_per_site); 0 = batch from blockIdx.z
+  int rem_ctas;      // 256 x 256 kernel: CTAs that each take the last blocks of the contraction of several tiles
+  int tiles_m, tiles_n;  // 256 x 256 kernel: tile grid (its launch is one-dimensional)
   float* out_f32;    // EPI_Z: [batch][r][ld_out];  EPI_C: [m][ld_out]
   float* out2_f32;   // EPI_Z: optional second copy, same layout
   int64_t ld_out;
@@ -316,17 +318,49 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar, drained_bar;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag, issued_s;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tile = blockIdx.x;
-  const int n_tile = blockIdx.y / p.splits, split = blockIdx.y % p.splits;
-  const int m0 = m_tile * 256, n0 = n_tile * 256;
-  const int kb0 = split * p.kb_per_split;
-  const int kb1 = (kb0 + p.kb_per_split < p.k_blocks) ? kb0 + p.kb_per_split : p.k_blocks;
-  const int nkb = kb1 > kb0 ? kb1 - kb0 : 0;
+  // Work of this CTA.  The first tiles * splits CTAs each own one tile and one of the `splits` equal parts of the
+  // first splits * kb_per_split blocks of the contraction (m fastest, so neighbours share a B panel at the same k).
+  // The rem_ctas CTAs after them take what is left of the contraction, the same block range for every tile, each for
+  // the tiles t = j, j + rem_ctas, ... one after the other: they fill the SMs that tiles * splits leaves empty.
+  const int n_tiles = p.tiles_m * p.tiles_n;
+  const int n_main = n_tiles * p.splits;
+  const bool is_rem = (int)blockIdx.x >= n_main;
+  const int rem_j = (int)blockIdx.x - n_main;
+  const int slots = p.splits + (p.rem_ctas > 0 ? 1 : 0);  // partial tiles per output tile
+  struct Item {
+    int m0, n0, kb0, kb1, slot;
+    int64_t tile_lin;
+  };
+  auto item_at = [&](int it, Item& w) -> bool {
+    int tile, split;
+    if (!is_rem) {
+      if (it > 0) return false;
+      const int rest = (int)blockIdx.x / p.tiles_m;
+      tile = (rest / p.splits) * p.tiles_m + (int)blockIdx.x % p.tiles_m;  // n_tile * tiles_m + m_tile
+      split = rest % p.splits;
+      w.kb0 = split * p.kb_per_split;
+      const int end = p.rem_ctas > 0 ? p.splits * p.kb_per_split : p.k_blocks;
+      w.kb1 = (w.kb0 + p.kb_per_split < end) ? w.kb0 + p.kb_per_split : end;
+    } else {
+      tile = rem_j + it * p.rem_ctas;
+      if (tile >= n_tiles) return false;
+      split = p.splits;
+      w.kb0 = p.splits * p.kb_per_split;
+      w.kb1 = p.k_blocks;
+    }
+    if (w.kb1 < w.kb0) w.kb1 = w.kb0;
+    const int m_tile = tile % p.tiles_m, n_tile = tile / p.tiles_m;
+    w.m0 = m_tile * 256;
+    w.n0 = n_tile * 256;
+    w.slot = split;
+    w.tile_lin = (int64_t)m_tile * p.tiles_n + n_tile;
+    return true;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -334,6 +368,7 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       mbar_init(&empty_bar[s], 1);
     }
     mbar_init(&accum_bar, 1);
+    mbar_init(&drained_bar, 128);
     abort_flag = 0;
     issued_s = 0;
     fence_mbar_init();
@@ -355,55 +390,73 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       prefetch_tmap(&tmA);
       prefetch_tmap(&tmB);
-      for (int i = 0; i < nkb; ++i) {
-        const int stage = i % STAGES;
-        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp)) break;
-        mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
-        uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
-        uint8_t* b_dst = a_dst + A_BYTES;
-        const int kb = kb0 + i;
-        const int bz = kb / p.kb_per_site;
-        const int kcoord = (kb % p.kb_per_site) * BK;
+      int g = 0;  // blocks issued so far, over all items: the stage ring runs on across items
+      bool go = true;
+      Item w;
+      for (int it = 0; go && item_at(it, w); ++it) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb, ++g) {
+          const int stage = g % STAGES;
+          const uint32_t ph = (uint32_t)(g / STAGES) & 1u;
+          if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp)) {
+            go = false;
+            break;
+          }
+          mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+          uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_BYTES;
+          const int bz = kb / p.kb_per_site;
+          const int kcoord = (kb % p.kb_per_site) * BK;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tma_load_3d(a_dst + c * CHUNK, &tmA, &full_bar[stage], m0 + c * 64, kcoord, bz);
+          for (int c = 0; c < 4; ++c) tma_load_3d(a_dst + c * CHUNK, &tmA, &full_bar[stage], w.m0 + c * 64, kcoord, bz);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tma_load_3d(b_dst + c * CHUNK, &tmB, &full_bar[stage], n0 + c * 64, kcoord, bz);
-        issued_s = i + 1;
+          for (int c = 0; c < 4; ++c) tma_load_3d(b_dst + c * CHUNK, &tmB, &full_bar[stage], w.n0 + c * 64, kcoord, bz);
+          issued_s = g + 1;
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      for (int i = 0; i < nkb; ++i) {
-        const int stage = i % STAGES;
-        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        if (!mbar_wait(&full_bar[stage], ph, abortp)) break;
+      int g = 0;
+      bool go = true;
+      Item w;
+      for (int it = 0; go && item_at(it, w); ++it) {
+        // the accumulators of the previous item have been read out
+        if (it > 0 && !mbar_wait(&drained_bar, (uint32_t)(it - 1) & 1u, abortp)) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-        const uint32_t b_addr = a_addr + A_BYTES;
+        for (int kb = w.kb0; kb < w.kb1; ++kb, ++g) {
+          const int stage = g % STAGES;
+          const uint32_t ph = (uint32_t)(g / STAGES) & 1u;
+          if (!mbar_wait(&full_bar[stage], ph, abortp)) {
+            go = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_BYTES;
 #pragma unroll
-        for (int k16 = 0; k16 < BK / 16; ++k16) {
-          const uint64_t bdesc = smem_desc(b_addr + (uint32_t)k16 * 2048u, CHUNK, 1024u);
-          const uint32_t acc = (i | k16) != 0 ? 1u : 0u;
-          umma_bf16(tmem_base, smem_desc(a_addr + (uint32_t)k16 * 2048u, CHUNK, 1024u), bdesc, IDESC, acc);
-          umma_bf16(tmem_base + 256u, smem_desc(a_addr + 2u * CHUNK + (uint32_t)k16 * 2048u, CHUNK, 1024u), bdesc, IDESC, acc);
+          for (int k16 = 0; k16 < BK / 16; ++k16) {
+            const uint64_t bdesc = smem_desc(b_addr + (uint32_t)k16 * 2048u, CHUNK, 1024u);
+            const uint32_t acc = (kb != w.kb0 || k16 != 0) ? 1u : 0u;
+            umma_bf16(tmem_base, smem_desc(a_addr + (uint32_t)k16 * 2048u, CHUNK, 1024u), bdesc, IDESC, acc);
+            umma_bf16(tmem_base + 256u, smem_desc(a_addr + 2u * CHUNK + (uint32_t)k16 * 2048u, CHUNK, 1024u), bdesc, IDESC, acc);
+          }
+          umma_commit(&empty_bar[stage]);
         }
-        umma_commit(&empty_bar[stage]);
+        if (go) umma_commit(&accum_bar);
       }
-      umma_commit(&accum_bar);
     }
   } else {
     const int q = warp & 3;
     const int row = q * 32 + lane;  // row inside each 128-row half
     const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
-    const bool ok = mbar_wait(&accum_bar, 0u, abortp);
-    tc_fence_after();
-    const int tiles_n = gridDim.y / p.splits;
-    const int64_t tile_lin = (int64_t)m_tile * tiles_n + n_tile;
-    // With a split contraction every CTA stores its partial tile and gemm256_reduce sums them in split
-    // order; otherwise the tile goes straight to C.
-    float* my_partial = p.splits > 1 ? p.partial + (tile_lin * p.splits + split) * (int64_t)(256 * 256) : nullptr;
-    if (ok) {
+    Item w;
+    for (int it = 0; item_at(it, w); ++it) {
+      if (!mbar_wait(&accum_bar, (uint32_t)it & 1u, abortp)) break;
+      tc_fence_after();
+      const int nkb = w.kb1 - w.kb0;
+      // With several partial tiles per output tile every CTA stores its own and gemm256_reduce sums them in slot order;
+      // otherwise the tile goes straight to C.
+      float* my_partial = slots > 1 ? p.partial + (w.tile_lin * slots + w.slot) * (int64_t)(256 * 256) : nullptr;
 #pragma unroll 1
       for (int c = 0; c < 32; ++c) {  // chunk c: half c / 16 of the tile, columns (c % 16) * 16 .. +15
         const int half = c / 16, col = (c % 16) * 16;
@@ -419,21 +472,24 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         } else {
-          const int64_t gm = (int64_t)m0 + half * 128 + row;
+          const int64_t gm = (int64_t)w.m0 + half * 128 + row;
           if (gm < p.m_extent) {
-            float* dst = p.out_f32 + gm * p.ld_out + n0 + col;
-            if (n0 + col + 16 <= p.n_extent && (p.ld_out & 3) == 0) {
+            float* dst = p.out_f32 + gm * p.ld_out + w.n0 + col;
+            if (w.n0 + col + 16 <= p.n_extent && (p.ld_out & 3) == 0) {
 #pragma unroll
               for (int i = 0; i < 4; ++i)
                 reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
             } else {
 #pragma unroll
               for (int i = 0; i < 16; ++i)
-                if (n0 + col + i < p.n_extent) dst[i] = v[i];
+                if (w.n0 + col + i < p.n_extent) dst[i] = v[i];
             }
           }
         }
       }
+      // this thread's part of the accumulators is in registers or memory: the next item may overwrite them
+      tc_fence_before();
+      mbar_arrive(&drained_bar);
     }
   }
 
@@ -649,6 +705,26 @@ GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch) {
   if (splits < 1) splits = 1;
   const int64_t per = ceil_div(g.k_blocks, splits);
   g.splits = (int)ceil_div(g.k_blocks, per);  // no empty split
+  g.kb_per_split = per;
+  g.rem_ctas = 0;
+  if (big) {
+    // SMs that tiles * splits leaves empty (64 tiles x 2 splits: 20 of 148) take the tail of every tile's contraction,
+    // each for ceil(tiles / R) tiles in turn.  Balance: a CTA of the main part runs kb_main blocks and one epilogue, a
+    // remainder CTA tpr times (kb_rem blocks and an epilogue); the epilogue and the refill of the pipeline are put at
+    // the time of 30 blocks (measured on the 1024 x 4096 gradient over 65 536 rows: 0 / 12 / 30 / 60 / 100 blocks give
+    // 383 / 370 / 369 / 373 / 376 us, 378 us without remainder CTAs -- the 20 extra SMs buy 2.4 %, not their 13.5 %
+    // share: with every SM multiplying the clock settles lower under the power limit).
+    const int64_t R = 148 - g.tiles * g.splits;
+    if (R >= 8) {
+      const int64_t tpr = ceil_div(g.tiles, R), ovh = 30;
+      const int64_t kb_rem = (g.k_blocks - g.splits * (tpr - 1) * ovh) / (g.splits * tpr + 1);
+      const int64_t kb_main = ceil_div(g.k_blocks - kb_rem, g.splits);
+      if (kb_rem >= 32 && g.k_blocks - g.splits * kb_main >= 16) {
+        g.rem_ctas = (int)R;
+        g.kb_per_split = kb_main;
+      }
+    }
+  }
   return g;
 }
 
@@ -687,7 +763,10 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
   p.kb_per_site = g.batch > 1 ? 0 : (int)g.kb_per_site;  // batched: one site per entry, the entry from blockIdx.z
   p.k_blocks = (int)g.k_blocks;
   p.splits = g.splits;
-  p.kb_per_split = (int)ceil_div(g.k_blocks, g.splits);
+  p.kb_per_split = (int)g.kb_per_split;
+  p.rem_ctas = g.rem_ctas;
+  p.tiles_m = (int)ceil_div(hx, g.bm);
+  p.tiles_n = (int)ceil_div(hy, g.bn);
   p.out_f32 = C;
   p.ld_out = hy;
   p.out_batch_stride = hx * hy;
@@ -696,11 +775,13 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
   p.status = status;
   dim3 grid((unsigned)ceil_div(hx, g.bm), (unsigned)(ceil_div(hy, g.bn) * g.splits), (unsigned)g.batch);
   if (g.bm == 256) {
-    cudaError_t err = launch_gemm256<kGemm256BK, kGemm256Stages>(tmX, tmY, p, grid, st);
-    if (err != cudaSuccess || g.splits == 1) return err;
+    const int slots = g.splits + (g.rem_ctas > 0 ? 1 : 0);
+    const dim3 grid1((unsigned)(g.tiles * g.splits + g.rem_ctas), 1, 1);
+    cudaError_t err = launch_gemm256<kGemm256BK, kGemm256Stages>(tmX, tmY, p, grid1, st);
+    if (err != cudaSuccess || slots == 1) return err;
     const int64_t quads = hx * hy / 4;
     unsigned blocks = (unsigned)(quads / 256 < 148 * 8 ? ceil_div(quads, 256) : 148 * 8);
-    DAD_LAUNCH(err, "gemm_tn_reduce", gemm256_reduce_kernel, blocks, 256, 0, st, (const float*)partial, g.splits, (int)hx,
+    DAD_LAUNCH(err, "gemm_tn_reduce", gemm256_reduce_kernel, blocks, 256, 0, st, (const float*)partial, slots, (int)hx,
                (int)hy, C);
     return err;
   }

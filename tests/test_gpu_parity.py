@@ -163,6 +163,27 @@ def test_full_grad_long_contraction(oracle, B, S, N, h_in, h_out):
     assert rel(grads[0].double().numpy(), oracle.full_grad(A, D)) <= 1e-4
 
 
+def test_full_grad_with_remainder_ctas(oracle, B):
+    """40 tiles of 256 x 256 in 3 splits leave 28 SMs without a CTA; those take the tail of every tile's contraction,
+    two tiles each in turn (a fourth partial tile per output tile).  Sampled output rows against the oracle, and two
+    runs bit for bit."""
+    dev = torch.device("cuda:0")
+    S, N, h_in, h_out = 5, 6144, 512, 5120     # 480 blocks of 64 rows: 3 x 142 in the main part, 54 in the tail
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 4111, torch.bfloat16, dev)
+    L = B.make_layer(A, D)
+    ws = B.new_workspace(B.dad_workspace_bytes(L, 1, 0), dev)
+    grads = []
+    for _ in range(2):
+        grad = torch.full((h_in, h_out), float("nan"), device=dev)
+        B.dad_full_grad(L, A, D, grad, None, ws)
+        B.dad_check(ws)
+        grads.append(grad.cpu())
+    assert torch.equal(grads[0], grads[1])
+    rows = [0, 255, 256, 300, 511]
+    ref = oracle.full_grad(A[:, :, rows].cpu(), D.cpu())
+    assert rel(grads[0][rows].double().numpy(), ref) <= 1e-4
+
+
 @pytest.mark.parametrize("h_in,h_out,K,batch", [(1024, 1024, 256, 16), (264, 520, 40, 3), (70, 50, 12, 2)])
 def test_reconstruct_batched_is_the_per_layer_sum_of_outer_products(oracle, B, h_in, h_out, K, batch):
     """Algorithm 1's P^T Q step for several layers of one shape in one call: every entry against the oracle's
