@@ -4,13 +4,13 @@
 //
 //   Gram:      8 x 8 tiles of the lower triangle of slab slab^T, four columns per MMA; row blocks are
 //              paired (i, nb-1-i) over the warps so that every warp owns about the same number of tiles;
-//   Cholesky:  panels of four columns, four threads per row.  Thread q of a row brings panel entry q
-//              up to date (a dot product over the columns already factored, four partial sums); after a
-//              barrier every row's threads factor their own copy of the 4 x 4 diagonal block in
-//              registers.  The reciprocal square root of a pivot starts before the decisions on that
-//              pivot (floor, zeroing rule -- the same as in orth.cu) are known and is replaced afterwards
-//              if they say so: the dependent chain is one reciprocal square root, one product and one
-//              fused multiply-add per column;
+//   Cholesky:  panels of four columns, two threads per row on the first four warps.  A thread brings two
+//              panel entries of its row up to date (dot products over the columns already factored,
+//              four partial sums each); after a barrier every row's threads factor their own copy of
+//              the 4 x 4 diagonal block in registers.  The reciprocal square root of a pivot starts
+//              before the floor test on that pivot is known (the test compares bit patterns, off the
+//              fp64 pipe) and is replaced afterwards if the test says so; floor and zeroing rule are
+//              those of orth.cu;
 //   solve:     rows <- L^{-1} rows as block forward substitution in product form,
 //              X_b = sum_{k<=b} M_bk Src_k with M_bb = L_bb^{-1}, M_bk = -L_bb^{-1} L_bk, Src_k = X_k
 //              (already solved, read back in fp32) for k < b and the unsolved rows for k = b; every warp
