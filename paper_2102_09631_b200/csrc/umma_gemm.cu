@@ -209,7 +209,55 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       finish = last_flag != 0;
       if (finish) __threadfence();
     }
-    if (finish) {
+    if constexpr (EPI == EPI_YT) {
+      // Y^T planes: thread `row` holds one row of the tile, but a plane row (fixed j) is contiguous along the tile's
+      // rows.  The tile is turned in shared memory -- the stages are free once the accumulator is complete -- and
+      // written out in 16-byte pieces (rows_dot at r = 64: 16 stores per thread instead of 128 two-byte ones).
+      static_assert(2 * BN * 128 * 2 <= STAGES * STAGE_BYTES, "the staging tile has to fit in the stages");
+      __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(smem);  // [plane][j][128 rows]
+      if (finish) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 16; ++c) {
+          float v[16];
+          if (nkb > 0) {
+            tmem_ld16(lane_base + c * 16, v);
+            if constexpr (MMA_N > BN) {
+              float w[16];
+              tmem_ld16(lane_base + BN + c * 16, w);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v[i] += w[i];
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int j = c * 16 + i;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v[i]);
+            stg[j * 128 + row] = hi;
+            stg[(BN + j) * 128 + row] = __float2bfloat16_rn(v[i] - __bfloat162float(hi));
+          }
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");  // all four epilogue warps, whatever they decided above
+      if (finish && p.out_planes) {
+        const int et = (warp - 2) * 32 + lane, seg = et & 15;
+        const int r = p.n_extent;
+        const int64_t g0 = (int64_t)m0 + seg * 8;  // first of the eight tile rows of this piece
+        for (int o = et >> 4; o < 2 * r; o += 8) {
+          const int plane = o >= r ? 1 : 0, j = o - plane * r;
+          const __nv_bfloat16* src = stg + (plane * BN + j) * 128 + seg * 8;
+          __nv_bfloat16* dst = p.out_planes + (((int64_t)batch * 2 + plane) * p.plane_rows + j) * p.ld_planes + g0;
+          if (g0 + 8 <= p.m_extent && (p.ld_planes & 7) == 0) {
+            *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+          } else {
+            for (int e = 0; e < 8; ++e)
+              if (g0 + e < p.m_extent) dst[e] = src[e];
+          }
+        }
+      }
+    } else if (finish) {
       const int64_t gm = (int64_t)m0 + row;  // global row of D
 #pragma unroll 1
       for (int c = 0; c < BN / 16; ++c) {
