@@ -27,7 +27,8 @@ if ROOT not in sys.path:
 # capture of each kernel on the 1024-wide layers of this workload (536.9 MB per launch).  DRAM traffic of these
 # streaming kernels grows in proportion to the slices a launch covers, so the ratio carries over to the larger
 # launches timed here.  Set an entry to None when its kernel changes until the counters are taken again.
-# cols_acc_tc: its 2048-CTA launches now take a two-stage form that has not been captured (1.043 for the five-stage one).
+# rows_dot_tc: recaptured after its epilogue change (1.040 / 1.038).  cols_acc_tc: its 2048-CTA launches now take a
+# two-stage form that has not been captured (1.043 for the five-stage one).
 DRAM_TRAFFIC_OVER_ALGORITHMIC = {"rows_dot_tc": 1.039, "cols_acc_tc": None}
 
 METRIC = "rank-dAD compress+reconstruct layers/s"
