@@ -54,6 +54,9 @@ def parse_args():
                     help="one call per layer instead of stacking the same-shape layers of a block into one call")
     ap.add_argument("--cuda-graph", action="store_true",
                     help="capture one step in a CUDA graph and time its replays (for launch-bound configurations)")
+    ap.add_argument("--streams", type=int, default=None,
+                    help="CUDA streams the independent calls of a step are dealt over (default: 3 for the launch-bound "
+                         "configurations 1-3, whose calls use a fraction of the GPU each; 1 for configurations 4-5)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -265,13 +268,26 @@ def run_ours(args):
             plans[key] = B.LayerPlan(A, D, r, iters, groups=groups)
     input_bytes = sum(A.numel() * A.element_size() + D.numel() * D.element_size() for blk in data for A, D, _ in blk)
     stream = torch.cuda.current_stream()
+    # Calls on different plans are independent (own inputs, workspace and outputs).  Where one call cannot fill the GPU
+    # the plans are dealt over several streams, each plan always on the same one; every step forks from and joins the
+    # timed stream, so the events around the timed region see all of the work.
+    n_streams = args.streams if args.streams is not None else (3 if cfg.index <= 3 else 1)
+    n_streams = 1 if args.cuda_graph else max(1, min(n_streams, len(plans)))
+    side_streams = [torch.cuda.Stream(device=dev) for _ in range(n_streams - 1)]
+    lane_of = {key: i % n_streams for i, key in enumerate(plans)}
 
     def step():
+        lanes = [stream] + side_streams
+        for sd in side_streams:
+            sd.wait_stream(stream)
         for b in range(n_super):
             blk = data[b % RB]
             for ui, (sh, groups) in enumerate(units):
                 A, D, Q0 = blk[ui]
-                plans[(sh.h_in, sh.h_out, groups)].step(A, D, Q0, stream)
+                key = (sh.h_in, sh.h_out, groups)
+                plans[key].step(A, D, Q0, lanes[lane_of[key]])
+        for sd in side_streams:
+            stream.wait_stream(sd)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -484,7 +500,9 @@ def run_ours(args):
                            "calls": ("one call per layer" if args.no_group else
                                      f"same-shape layers of {G} consecutive block(s) stacked as extra slices of one call: " +
                                      ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
-                           "launch": "CUDA graph replay" if args.cuda_graph else "stream launches",
+                           "launch": "CUDA graph replay" if args.cuda_graph else
+                                     ("stream launches" if n_streams == 1 else
+                                      f"stream launches, the step's independent calls dealt over {n_streams} streams"),
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
                 "kernels": kernels, "reconstruct": reconstruct, "dad_full_grad": full_grad, "compulsory_traffic": compulsory,
