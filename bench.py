@@ -272,7 +272,7 @@ def run_ours(args):
     # the plans are dealt over several streams, each plan always on the same one; every step forks from and joins the
     # timed stream, so the events around the timed region see all of the work.
     n_streams = args.streams if args.streams is not None else (3 if cfg.index <= 3 else 1)
-    n_streams = 1 if args.cuda_graph else max(1, min(n_streams, len(plans)))
+    n_streams = max(1, min(n_streams, len(plans)))
     side_streams = [torch.cuda.Stream(device=dev) for _ in range(n_streams - 1)]
     lane_of = {key: i % n_streams for i, key in enumerate(plans)}
 
@@ -500,9 +500,9 @@ def run_ours(args):
                            "calls": ("one call per layer" if args.no_group else
                                      f"same-shape layers of {G} consecutive block(s) stacked as extra slices of one call: " +
                                      ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
-                           "launch": "CUDA graph replay" if args.cuda_graph else
-                                     ("stream launches" if n_streams == 1 else
-                                      f"stream launches, the step's independent calls dealt over {n_streams} streams"),
+                           "launch": ("CUDA graph replay" if args.cuda_graph else "stream launches") +
+                                     ("" if n_streams == 1 else
+                                      f", the step's independent calls dealt over {n_streams} streams"),
                            "factors": "fp32", "accumulate": "f64" if cfg.dtype == "f32" else "f32"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
                 "kernels": kernels, "reconstruct": reconstruct, "dad_full_grad": full_grad, "compulsory_traffic": compulsory,
