@@ -189,7 +189,7 @@ dad_status dad_gather_factors(const dad_layer* layer, int r, const float* P, con
  *              16 significant bits of the factors (the dropped lo*lo term is 2^-16 relative).
  *              Needs h_in and h_out multiples of 8; otherwise DAD_BF16 falls back to the
  *              fp32 FMA kernel (still on the device).
- *   ws         DEVICE scratch of ws_bytes >= dad_reconstruct_workspace_bytes(h_in, h_out, K),
+ *   ws         DEVICE scratch of ws_bytes >= dad_reconstruct_workspace_bytes(h_in, h_out, K, math),
  *              may be NULL when that is 0
  */
 size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math);
@@ -270,8 +270,11 @@ dad_status dad_effective_rank(const dad_layer* layer, int r, float theta, const 
  * cudaMalloc/cudaFree and calls no allocating library routine.
  *   - Problems whose scratch need (dad_reconstruct_workspace_bytes) exceeds
  *     DAD_STATIC_SCRATCH_BYTES are refused with DAD_ERR_WORKSPACE; nothing is launched.
- *   - The first call on each device resolves the array's device address (and clears its status
- *     words on `cuda_stream`); make that first call outside any stream capture.
+ *   - The first call on each device resolves the array's device address.  That is also the moment
+ *     the CUDA runtime loads the module holding the array, i.e. when its DAD_STATIC_SCRATCH_BYTES
+ *     are taken from that device (with the device-wide synchronisation a module load implies, and
+ *     DAD_ERR_CUDA if the device has no room left); only the calls after it leave the device's
+ *     memory untouched.  Make that first call early, and outside any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents; the
  *     library clears what has to start at zero.  Two calls that overlap in time on the same GPU
  *     (different streams, different host threads) race on it: serialise them, or use dad_reconstruct

@@ -30,6 +30,16 @@ static dad_status validate_layer(const dad_layer* L) {
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// With one site the header leaves the site strides unspecified; every internal user gets N * ld instead.
+static dad_layer normalised(const dad_layer& in) {
+  dad_layer L = in;
+  if (L.S == 1) {
+    L.strideA = L.N * L.ldA;
+    L.strideD = L.N * L.ldD;
+  }
+  return L;
+}
+
 bool tc_eligible(const dad_layer& L) {
   if (L.dtype != DAD_BF16) return false;
   if ((L.h_in | L.h_out | L.ldA | L.ldD) % 8 != 0) return false;
@@ -283,18 +293,22 @@ static dad_status validate_rank(const dad_layer* L, int r) {
   return DAD_OK;
 }
 
-size_t dad_workspace_bytes(const dad_layer* L, int r, int iters) {
-  if (validate_layer(L) != DAD_OK || validate_rank(L, r) != DAD_OK || iters < 0) return 0;
+size_t dad_workspace_bytes(const dad_layer* layer, int r, int iters) {
+  if (validate_layer(layer) != DAD_OK || validate_rank(layer, r) != DAD_OK || iters < 0) return 0;
+  const dad_layer Ln = normalised(*layer);
+  const dad_layer* L = &Ln;
   const bool tc = tc_eligible(*L);
   const size_t a = compress_ws_layout(*L, r, L->dtype == DAD_F32, tc).total;
   const size_t b = tc ? gemm_ws_layout(L->h_in, L->h_out, L->S, L->N, false).total : 256;
   return a > b ? a : b;
 }
 
-dad_status dad_full_grad(const dad_layer* L, const void* A, const void* D, float* grad, uint64_t* bytes_tx,
+dad_status dad_full_grad(const dad_layer* layer, const void* A, const void* D, float* grad, uint64_t* bytes_tx,
                          void* ws, size_t ws_bytes, void* cuda_stream) {
-  dad_status vs = validate_layer(L);
+  dad_status vs = validate_layer(layer);
   if (vs != DAD_OK) return vs;
+  const dad_layer Ln = normalised(*layer);
+  const dad_layer* L = &Ln;
   if (!A || !D || !grad) return DAD_ERR_NULL;
   if (!aligned(A, 16) || !aligned(D, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -314,10 +328,12 @@ dad_status dad_full_grad(const dad_layer* L, const void* A, const void* D, float
   return DAD_OK;
 }
 
-dad_status dad_rank_compress(const dad_layer* L, const void* A, const void* D, int r, int iters, const float* Q0,
+dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* D, int r, int iters, const float* Q0,
                              float* P, float* Q, float* sigma, void* ws, size_t ws_bytes, void* cuda_stream) {
-  dad_status vs = validate_layer(L);
+  dad_status vs = validate_layer(layer);
   if (vs != DAD_OK) return vs;
+  const dad_layer Ln = normalised(*layer);
+  const dad_layer* L = &Ln;
   if (!A || !D || !Q0 || !P || !Q || !ws) return DAD_ERR_NULL;
   vs = validate_rank(L, r);
   if (vs != DAD_OK) return vs;

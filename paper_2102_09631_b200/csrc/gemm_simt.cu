@@ -195,7 +195,7 @@ cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16
   return err;
 }
 
-// Operands of the reconstruction sum_k P_k^T Q_k (Section 3.4) for a bf16 tensor-core product that keeps
+// Operands of the reconstruction sum_k P_k^T Q_k (Algorithm 1, the P^T Q step; Section 3.3) for a bf16 tensor-core product that keeps
 // fp32-level accuracy: with x = hi(x) + lo(x) (two bf16 terms), P^T Q ~= hi^T hi + hi^T lo + lo^T hi, the
 // dropped lo^T lo term being 2^-16 relative.  The three products become one contraction of length 3K over
 //     X3 = [hi(P); hi(P); lo(P)]   and   Y3 = [hi(Q); lo(Q); hi(Q)].

@@ -68,6 +68,11 @@ dad_status dad_rank_dad_host(const dad_layer* layer, const void* A_host, const v
   if (!layer || !A_host || !D_host || !Q0_host || !grad_host || !dev_scratch) return DAD_ERR_NULL;
   if (math != DAD_F32 && math != DAD_BF16) return DAD_ERR_DTYPE;
   if (reinterpret_cast<uintptr_t>(dev_scratch) % 256) return DAD_ERR_ALIGN;
+  // the caller's own strides feed the copies: rows must not overlap, sites must not overlap (before anything is queued)
+  if (layer->S >= 1 && layer->N >= 1 && layer->h_in >= 1 && layer->h_out >= 1) {
+    if (layer->ldA < layer->h_in || layer->ldD < layer->h_out) return DAD_ERR_SHAPE;
+    if (layer->S > 1 && (layer->strideA < layer->N * layer->ldA || layer->strideD < layer->N * layer->ldD)) return DAD_ERR_SHAPE;
+  }
   HostScratch sc;
   if (!carve(*layer, r, iters, math, &sc)) {
     // let the device entry point name the reason (shape, dtype, rank) without touching memory

@@ -7,7 +7,9 @@
 // allocation brings.  dad_reconstruct on the tensor cores needs scratch (bf16 copies of the two
 // factor stacks, split partial tiles, counters); here that scratch is a fixed array that lives in
 // the library's device image, so the call allocates nothing -- at the price of 32 MiB held on every
-// GPU that loads the library, for as long as the process lives.
+// GPU that loads the library, for as long as the process lives.  (The first call on a device makes the
+// runtime load the module that holds the array, which is when those 32 MiB are taken; later calls
+// change nothing in the device's memory.)
 #include <mutex>
 
 #include "common.cuh"
@@ -23,7 +25,10 @@ std::mutex g_mu;
 void* g_scratch_ptr[kMaxDevices] = {nullptr};
 
 // Device address of the scratch array on the current device, resolved once per device.
-cudaError_t scratch_for_current_device(void** out, cudaStream_t st) {
+// The first call on a device is also where the CUDA runtime loads this translation unit's module, which is when the
+// array's 32 MiB are reserved on that device; a __device__ array starts out zeroed, so the status words at its head
+// need no clearing.
+cudaError_t scratch_for_current_device(void** out) {
   int dev = -1;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
@@ -32,9 +37,6 @@ cudaError_t scratch_for_current_device(void** out, cudaStream_t st) {
   if (!g_scratch_ptr[dev]) {
     void* p = nullptr;
     err = cudaGetSymbolAddress(&p, g_static_scratch);
-    if (err != cudaSuccess) return err;
-    // the status words at the head of a workspace must start out clear
-    err = cudaMemsetAsync(p, 0, 256, st);
     if (err != cudaSuccess) return err;
     g_scratch_ptr[dev] = p;
   }
@@ -52,7 +54,7 @@ extern "C" dad_status dad_reconstruct_static(int64_t h_in, int64_t h_out, int64_
   if (need > (size_t)DAD_STATIC_SCRATCH_BYTES) return DAD_ERR_WORKSPACE;  // larger problems: dad_reconstruct with caller scratch
   void* scratch = nullptr;
   if (need > 0) {
-    if (scratch_for_current_device(&scratch, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    if (scratch_for_current_device(&scratch) != cudaSuccess)
       return DAD_ERR_CUDA;
   }
   return dad_reconstruct(h_in, h_out, K, Pcat, Qcat, grad, math, scratch, need > 0 ? (size_t)DAD_STATIC_SCRATCH_BYTES : 0,

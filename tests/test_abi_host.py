@@ -68,6 +68,12 @@ def test_workspace_query(B):
     assert B.dad_workspace_bytes(L, 4, -1) == 0
     assert B.dad_workspace_bytes(layer(B, dtype=7), 4, 2) == 0
     assert B.dad_workspace_bytes(layer(B, N=4096, h_in=1024, h_out=4096, dtype=1, S=16), 64, 3) >= n
+    # one site: the site strides are unspecified and must not matter (odd, zero or huge values)
+    one = dict(S=1, N=64, h_in=128, h_out=256, dtype=1, ldA=128, ldD=256)
+    ref = B.dad_workspace_bytes(layer(B, strideA=64 * 128, strideD=64 * 256, **one), 8, 2)
+    assert ref > 0
+    for sa, sd in ((0, 0), (3, 5), (1 << 50, 1 << 50)):
+        assert B.dad_workspace_bytes(layer(B, strideA=sa, strideD=sd, **one), 8, 2) == ref
 
 
 def test_bad_arguments_are_rejected_before_any_launch(B):
@@ -106,6 +112,13 @@ def test_bad_arguments_are_rejected_before_any_launch(B):
     assert lib.dad_reconstruct_batched_workspace_bytes(4, 4, 4, 0, 1) == 0
     assert lib.dad_gather_factors(ctypes.byref(L), 0, p, p, p, p, None, None) == E["DAD_ERR_RANK"]
     assert lib.dad_check(null, None) == E["DAD_ERR_NULL"]
+    # host entry point: the caller's own row and site strides are checked before any copy is queued
+    def host(Lx, scratch=p, nbytes=1 << 40):
+        return lib.dad_rank_dad_host(ctypes.byref(Lx), p, p, p, 4, 2, 0, p, None, scratch, nbytes, None)
+    assert host(layer(B, ldA=63)) == E["DAD_ERR_SHAPE"]
+    assert host(layer(B, ldD=31)) == E["DAD_ERR_SHAPE"]
+    assert host(layer(B, strideA=16 * 64 - 1)) == E["DAD_ERR_SHAPE"]
+    assert host(layer(B), scratch=ctypes.c_void_p(0x10100), nbytes=256) == E["DAD_ERR_WORKSPACE"]
     assert B.dad_launch_count() == before
     for code in range(len(B.STATUS_NAMES)):
         assert len(lib.dad_status_string(code)) > 0
