@@ -135,6 +135,24 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
                              void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Which of the library's pipelines dad_rank_compress takes for this shape (informational; the paper has no
+ * counterpart).  All three compute the iteration stated above to the same precision contract:
+ *   DAD_PATH_GENERAL  any shape: one launch per product and per Cholesky-QR phase (5 * iters + 3 or more launches)
+ *   DAD_PATH_TENSOR   bf16 inputs in 16-byte-aligned layouts: the same sequence on tcgen05 tensor cores
+ *   DAD_PATH_FUSED    small sites: ONE launch, a thread-block cluster of *cluster_size CTAs per site runs every
+ *                     application of the operator, the orthonormalisations and the final factor, with Y and W
+ *                     in shared memory and the partial sums of Z and G~ exchanged inside the cluster.
+ * Returns -1 for invalid arguments; cluster_size may be NULL.  dad_fused_enable(0) makes the library skip the
+ * one-launch form (process-wide; for timing one pipeline against the other), dad_fused_enable(1) restores it.
+ * The workspace size does not depend on that switch.
+ */
+#define DAD_PATH_GENERAL 0
+#define DAD_PATH_TENSOR 1
+#define DAD_PATH_FUSED 2
+int dad_compress_path(const dad_layer* layer, int r, int iters, int* cluster_size);
+void dad_fused_enable(int on);
+
+/*
  * The same compression in the form Algorithm 2 prints it, for the regime the paper assumes (batch much smaller
  * than the layer width, N << h; Sec. 3.3.1): C = A A^T (N x N) is precomputed once per site, every application
  * of the operator then touches only D and C,  g <- D^T ( C ( D g ) )  (Eq. "reduced_iter" with B = D^T C), and

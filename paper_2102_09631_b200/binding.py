@@ -28,7 +28,7 @@ EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_b
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
            "dad_rank_compress_gram", "dad_rank_compress_sequential_workspace_bytes", "dad_rank_compress_sequential",
-           "dad_check", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
+           "dad_check", "dad_compress_path", "dad_fused_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
 
@@ -106,6 +106,10 @@ def lib() -> ctypes.CDLL:
         L.dad_rank_compress_sequential.argtypes = [lp, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp,
                                                    ctypes.c_size_t, vp]
         L.dad_rank_compress_sequential.restype = ctypes.c_int
+        L.dad_compress_path.argtypes = [lp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+        L.dad_compress_path.restype = ctypes.c_int
+        L.dad_fused_enable.argtypes = [ctypes.c_int]
+        L.dad_fused_enable.restype = None
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -173,6 +177,19 @@ def dad_bytes_dsgd(layer: dad_layer) -> int:
 
 def dad_workspace_bytes(layer: dad_layer, r: int, iters: int) -> int:
     return int(lib().dad_workspace_bytes(ctypes.byref(layer), r, iters))
+
+
+DAD_PATH_GENERAL, DAD_PATH_TENSOR, DAD_PATH_FUSED = 0, 1, 2
+
+
+def dad_compress_path(layer: dad_layer, r: int, iters: int):
+    """(path, cluster size) dad_rank_compress takes for this shape; path is one of DAD_PATH_*."""
+    c = ctypes.c_int(0)
+    return int(lib().dad_compress_path(ctypes.byref(layer), r, iters, ctypes.byref(c))), c.value
+
+
+def dad_fused_enable(on: bool):
+    lib().dad_fused_enable(1 if on else 0)
 
 
 def dad_launch_count() -> int:

@@ -8,6 +8,7 @@
 namespace dad {
 
 std::atomic<uint64_t> g_launches{0};
+static std::atomic<bool> g_fused_on{true};
 
 static bool layer_ok(const dad_layer* L) {
   if (!L) return false;
@@ -48,7 +49,7 @@ bool tc_eligible(const dad_layer& L) {
   return tmap_encoder_available();
 }
 
-CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc) {
+CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc, int fused_c) {
   CompressWs w;
   memset(&w, 0, sizeof(w));
   const size_t acc = f64 ? 8 : 4;
@@ -61,11 +62,11 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc) {
   w.counters = off;
   off = align_up(off + w.n_counters * sizeof(unsigned), 256);
   w.G = off;
-  off = align_up(off + (f64 ? S * rr * ho * acc : 0), 256);
+  off = align_up(off + ((f64 || fused_c > 0) ? S * rr * ho * acc : 0), 256);
   w.Y = off;
   off = align_up(off + (tc ? 0 : S * N * rr * acc), 256);
   w.Z = off;
-  off = align_up(off + (tc ? 0 : S * rr * hi * acc), 256);
+  off = align_up(off + ((tc && fused_c == 0) ? 0 : S * rr * hi * acc), 256);
   size_t part = 0;
   if (!tc) {
     const int s_in = cols_acc_splits(L.S, L.N, L.h_in), s_out = cols_acc_splits(L.S, L.N, L.h_out);
@@ -96,6 +97,13 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc) {
     const size_t p_out = (size_t)umma_cols_acc_splits(L.S, L.N, L.h_out) * (size_t)ceil_div(L.h_out, 128);
     w.tc_partial = off;
     off = align_up(off + S * (p_in > p_out ? p_in : p_out) * 128 * rp * 4, 256);
+  }
+  w.fused_part = w.fused_sig = off;
+  if (fused_c > 0) {
+    w.fused_part = off;
+    off = align_up(off + S * (size_t)fused_c * rr * hmax * acc, 256);
+    w.fused_sig = off;
+    off = align_up(off + S * (size_t)fused_c * rr * 8, 256);
   }
   w.total = off;
   return w;
@@ -298,7 +306,7 @@ size_t dad_workspace_bytes(const dad_layer* layer, int r, int iters) {
   const dad_layer Ln = normalised(*layer);
   const dad_layer* L = &Ln;
   const bool tc = tc_eligible(*L);
-  const size_t a = compress_ws_layout(*L, r, L->dtype == DAD_F32, tc).total;
+  const size_t a = compress_ws_layout(*L, r, L->dtype == DAD_F32, tc, fused_cluster_size(*L, r, iters)).total;
   const size_t b = tc ? gemm_ws_layout(L->h_in, L->h_out, L->S, L->N, false).total : 256;
   return a > b ? a : b;
 }
@@ -343,11 +351,18 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
     return DAD_ERR_ALIGN;
   const bool f64 = L->dtype == DAD_F32;
   const bool tc = tc_eligible(*L);
-  const CompressWs w = compress_ws_layout(*L, r, f64, tc);
+  const int fused_c = fused_cluster_size(*L, r, iters);
+  const CompressWs w = compress_ws_layout(*L, r, f64, tc, fused_c);
   if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
-  if (tc)
+  if (fused_c > 0 && g_fused_on.load(std::memory_order_relaxed)) {
+    char* base = static_cast<char*>(ws);
+    err = cudaMemsetAsync(base + w.status, 0, 4, st);
+    if (err == cudaSuccess)
+      err = fused_compress(*L, A, D, r, iters, Q0, P, Q, sigma, base + w.G, base + w.Z, base + w.fused_part,
+                           reinterpret_cast<double*>(base + w.fused_sig), reinterpret_cast<int*>(base + w.status), fused_c, st);
+  } else if (tc)
     err = run_compress_tc(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st);
   else if (f64)
     err = run_compress<double>(*L, A, D, r, iters, Q0, P, Q, sigma, (char*)ws, w, st);
@@ -431,6 +446,20 @@ dad_status dad_check(const void* ws, void* cuda_stream) {
     if (status[i] == (int)DAD_ERR_TIMEOUT || status[i] == (int)DAD_ERR_NUMERIC) return (dad_status)status[i];
   return DAD_OK;
 }
+
+int dad_compress_path(const dad_layer* layer, int r, int iters, int* cluster_size) {
+  if (cluster_size) *cluster_size = 0;
+  if (validate_layer(layer) != DAD_OK || validate_rank(layer, r) != DAD_OK || iters < 0) return -1;
+  const dad_layer L = normalised(*layer);
+  const int c = g_fused_on.load(std::memory_order_relaxed) ? fused_cluster_size(L, r, iters) : 0;
+  if (c > 0) {
+    if (cluster_size) *cluster_size = c;
+    return DAD_PATH_FUSED;
+  }
+  return tc_eligible(L) ? DAD_PATH_TENSOR : DAD_PATH_GENERAL;
+}
+
+void dad_fused_enable(int on) { g_fused_on.store(on != 0, std::memory_order_relaxed); }
 
 uint64_t dad_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

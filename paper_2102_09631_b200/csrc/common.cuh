@@ -33,6 +33,23 @@ void timing_mark(const char* tag, cudaStream_t st, bool begin);
     if ((err) == cudaSuccess) (err) = e__;                                      \
   } while (0)
 
+// True the first time it is asked on each device (per object): for per-function set-up such as the opt-in to
+// large dynamic shared memory, which need not be repeated at every launch.
+struct FirstUse {
+  std::atomic<uint64_t> seen{0};
+  int last = -1;
+  bool on_this_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev > 63) return true;
+    last = dev;
+    const uint64_t bit = 1ull << dev;
+    return (seen.fetch_or(bit, std::memory_order_relaxed) & bit) == 0;
+  }
+  void forget() {
+    if (last >= 0) seen.fetch_and(~(1ull << last), std::memory_order_relaxed);
+  }
+};
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
@@ -66,10 +83,20 @@ struct CompressWs {
   size_t Yt;            // S*2*rp*Npad  bf16: planes of Y^T (operand of Y^T A and W^T D)
   int64_t Npad;
   size_t tc_partial;    // split partial tiles of the tensor-core column products
+  // one-launch compress: per-CTA partial sums S*C*r*max(h) of the accumulator type, slice lengths S*C*r doubles
+  size_t fused_part, fused_sig;
   size_t total;
 };
-// f64: fp64 pipeline (fp32 inputs); tc: tensor-core pipeline (bf16 inputs, 16-byte-aligned layout)
-CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc);
+// f64: fp64 pipeline (fp32 inputs); tc: tensor-core pipeline (bf16 inputs, 16-byte-aligned layout);
+// fused_c: cluster size of the one-launch compress (0: not used for this shape)
+CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc, int fused_c);
+
+// One-launch compress of small sites (fused_site.cu): a cluster of `C` CTAs per site runs the whole structured
+// power iteration.  fused_cluster_size gives C for a shape, or 0 when the multi-launch pipelines take it.
+int fused_cluster_size(const dad_layer& L, int r, int iters);
+cudaError_t fused_compress(const dad_layer& L, const void* A, const void* D, int r, int iters, const float* Q0, float* P,
+                           float* Q, float* sigma, void* FG, void* FZ, void* part, double* sig_part, int* status, int C,
+                           cudaStream_t st);
 
 // Workspace of dad_full_grad and of dad_reconstruct on the tensor cores.
 struct GemmWs {

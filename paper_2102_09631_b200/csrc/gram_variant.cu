@@ -81,7 +81,7 @@ struct GramWs {
 
 GramWs gram_ws_layout(const dad_layer& L, int r) {
   GramWs w;
-  w.base = compress_ws_layout(L, r, true, false);
+  w.base = compress_ws_layout(L, r, true, false, 0);
   size_t off = w.base.total;
   w.C = off;
   off = align_up(off + (size_t)L.S * L.N * L.N * 8, 256);

@@ -115,7 +115,7 @@ struct SeqWs {
 
 SeqWs seq_ws_layout(const dad_layer& L, int r) {
   SeqWs w;
-  w.base = compress_ws_layout(L, 1, true, false);
+  w.base = compress_ws_layout(L, 1, true, false, 0);
   size_t off = w.base.total;
   w.T = off;
   off = align_up(off + (size_t)L.S * L.h_out * 8, 256);

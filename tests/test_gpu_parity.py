@@ -81,6 +81,43 @@ def check_layer(oracle, B, A, D, Q0, r, iters, tol, ortho_tol=1e-4, compare_fact
     return g, o
 
 
+@pytest.mark.parametrize("S,N,h_in,h_out,r,iters,dtype", [
+    (2, 16, 64, 32, 4, 2, torch.float32),         # configuration 1
+    (4, 128, 1024, 1024, 8, 3, torch.float32),    # configuration 2, hidden layer: 8 CTAs per site, 16 rows each
+    (4, 128, 1024, 10, 8, 3, torch.float32),      # its output layer: fewer columns than CTAs in the cluster
+    (18, 64, 784, 1024, 8, 3, torch.float32),     # the paper's own setting: batch 64 per site, 18 sites
+    (1, 32, 784, 1024, 8, 3, torch.float32),      # the aggregator's stacks of a small layer as one site
+    (3, 70, 264, 520, 40, 2, torch.float32),      # large rank (8 x 8 register blocks in the Cholesky-QR), ragged rows
+    (5, 37, 50, 70, 7, 12, torch.float32),        # odd everything, many iterations
+    (2, 300, 256, 512, 16, 2, torch.bfloat16),    # bf16 inputs small enough for one cluster: fp32 accumulation
+    (3, 100, 70, 50, 7, 2, torch.bfloat16),
+])
+def test_one_launch_compress_matches_oracle_and_the_multi_launch_pipeline(oracle, B, S, N, h_in, h_out, r, iters, dtype):
+    """Shapes the one-launch compress takes (a cluster per site for the whole structured power iteration):
+    parity with the oracle at the usual bars, two runs bit for bit, and agreement with the multi-launch
+    pipeline on the same inputs (same subspace: the projected gradients agree far inside the bar)."""
+    dev = torch.device("cuda:0")
+    seed = 900 + N + h_in
+    A, D = wl.decaying_layer(S, N, h_in, h_out, seed, dtype)
+    Q0 = wl.start_block(S, r, h_out, seed)
+    path, C = B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)
+    assert path == B.DAD_PATH_FUSED and C >= 1
+    tol = TOL[dtype]
+    g1, o = check_layer(oracle, B, A, D, Q0, r, iters, tol, ortho_tol=1e-3 if dtype == torch.bfloat16 else 1e-4)
+    before = B.dad_launch_count()
+    g2 = run_gpu_layer(B, A, D, Q0, r, iters)
+    assert np.array_equal(g1["P"], g2["P"]) and np.array_equal(g1["Q"], g2["Q"]) and np.array_equal(g1["sigma"], g2["sigma"])
+    B.dad_fused_enable(False)
+    try:
+        assert B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)[0] != B.DAD_PATH_FUSED
+        g3 = run_gpu_layer(B, A, D, Q0, r, iters)
+    finally:
+        B.dad_fused_enable(True)
+    for s in range(S):
+        assert rel(g1["P"][s].T @ g1["Q"][s], g3["P"][s].T @ g3["Q"][s]) <= tol
+    assert rel(g1["grad"], g3["grad"]) <= tol
+
+
 def test_config1_single_linear_layer(oracle, B):
     cfg = wl.CONFIGS[1]
     A, D, Q0 = wl.layer_inputs(cfg, cfg.layers[0], 0)
