@@ -62,6 +62,11 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile-pass", action="store_true")
     ap.add_argument("--no-full-grad", action="store_true", help="skip timing the uncompressed dAD gradient")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the other configurations and the rank / iteration sweep of configuration 5 that a default "
+                         "run reports beside its headline workload")
+    ap.add_argument("--sweep-steps", type=int, default=3, help="timed steps of each sweep entry")
+    ap.add_argument("--no-check", action="store_true", help="skip the oracle check of one sampled site per workload")
     return ap.parse_args()
 
 
@@ -205,7 +210,17 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+def sweep_entries(args):
+    """(config, r, iters) of the workloads a default run reports beside the headline: configurations 1-4 as they are
+    defined, and configuration 5 over r in {4, 16, 64} x iters in {1, 3}."""
+    from paper_2102_09631_b200 import workloads as wl
+    out = [(c, wl.CONFIGS[c].r, wl.CONFIGS[c].iters) for c in (1, 2, 3, 4)]
+    out += [(5, r, it) for r in (4, 16, 64) for it in (1, 3)]
+    return out
+
+
 def run_ours(args):
+    import copy
     import torch
     import torch.distributed as dist
     from paper_2102_09631_b200 import binding as B, build as dad_build, multi, workloads as wl
@@ -218,6 +233,50 @@ def run_ours(args):
     multi.init("nccl", dev)
     dad_build.build()
     B.lib()
+    line = measure(args, rank, local, world, dev, headline=True)
+    default_workload = (args.config == 5 and args.rank is None and args.iters is None and args.blocks is None
+                        and not args.no_group and not args.cuda_graph and args.streams is None)
+    if default_workload and not args.no_sweep and world == 1:
+        sweep = []
+        for c, r, it in sweep_entries(args):
+            a = copy.copy(args)
+            a.config, a.rank, a.iters = c, r, it
+            a.no_e2e = a.no_cpu_baseline = a.no_full_grad = True
+            a.steps = args.sweep_steps if c >= 4 else 20      # the launch-bound configurations take well under a millisecond
+            a.warmup = max(3, args.warmup if c >= 4 else 10)
+            torch.cuda.empty_cache()
+            e = measure(a, rank, local, world, dev, headline=False)
+            if e is not None:
+                keep = ("ms_per_step", "value", "unit", "steps", "warmup", "gpu_launches", "launches_per_compress", "clocks",
+                        "roofline", "reconstruct", "stream_gbs", "check", "compress_path")
+                sweep.append({"config": c, "r": r, "iters": it, "workload": e["config"]["workload"],
+                              **{k: e.get(k) for k in keep}})
+        if line is not None:
+            line["sweep"] = sweep
+    if rank == 0 and line is not None:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def oracle_check(cfg, r, iters, plan, A, D, Q0, site=0):
+    """Relative Frobenius error of the projected gradient P_s^T Q_s of one site, as the library left it in the
+    plan's buffers, against the float64 oracle on the same inputs (the oracle as checker, outside every timed region)."""
+    import numpy as np
+    from oracle import dad_oracle
+    dad_oracle.build()
+    a, d, q0 = A[site:site + 1].cpu(), D[site:site + 1].cpu(), Q0[site:site + 1].cpu()
+    Po, Qo, _ = dad_oracle.spi_block(a, d, q0, iters)
+    ref = Po[0].T @ Qo[0]
+    got = plan.P[site].double().cpu().numpy().T @ plan.Q[site].double().cpu().numpy()
+    err = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
+    return {"site": site, "quantity": "P_s^T Q_s", "rel_frobenius_error": err,
+            "bar": 1e-5 if cfg.dtype == "f32" else 2e-2, "against": "float64 oracle, same inputs"}
+
+
+def measure(args, rank, local, world, dev, headline):
+    import torch
+    from paper_2102_09631_b200 import binding as B, multi, workloads as wl
 
     cfg = wl.CONFIGS[args.config]
     if args.blocks is not None:
@@ -355,6 +414,10 @@ def run_ours(args):
         base = "rows_dot" if name.startswith("rows_dot") else "cols_acc" if name.startswith("cols_acc") else None
         if base:
             alg = sum(stream_bytes_per_layer(cfg, sh, iters)[base] for sh in layers) * cfg.blocks * psteps
+        elif name.startswith("fused_site"):
+            # the one-launch compress makes every pass over A and Delta itself: all of the streamed bytes
+            alg = sum(stream_bytes_per_layer(cfg, sh, iters)[b] for sh in layers for b in ("rows_dot", "cols_acc")) \
+                  * cfg.blocks * psteps
         if alg and n:
             achieved = alg / (tms * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -472,6 +535,25 @@ def run_ours(args):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                "call": "dad_rank_dad_host per layer (host A, Delta, Q0 in; host gradient out), layers alternate over two streams"}
 
+    # ---- launches of one compress call, the pipeline each plan takes, and one sampled site against the oracle ----
+    sh0, groups0 = units[0]
+    key0 = (sh0.h_in, sh0.h_out, groups0)
+    A0, D0, Q00 = data[(n_super - 1) % RB][0]          # what the plan of the first unit saw last
+    plan0 = plans[key0]
+    torch.cuda.synchronize()
+    c0 = B.dad_launch_count()
+    B.dad_rank_compress(plan0.layer, A0, D0, r, iters, Q00, plan0.P, plan0.Q, plan0.sigma, plan0.ws, stream)
+    torch.cuda.synchronize()
+    launches_per_compress = B.dad_launch_count() - c0
+    names = {B.DAD_PATH_GENERAL: "general", B.DAD_PATH_TENSOR: "tensor", B.DAD_PATH_FUSED: "fused",
+             B.DAD_PATH_FUSED_L2: "fused_l2"}
+    compress_path = {f"{k[0]}->{k[1]} x{k[2]}": names.get(B.dad_compress_path(pl.layer, r, iters)[0], "?")
+                     for k, pl in plans.items()}
+    check = None
+    if rank == 0 and not args.no_check:
+        check = oracle_check(cfg, r, iters, plan0, A0, D0, Q00)
+        check["layer"] = f"{sh0.h_in}->{sh0.h_out}"
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import dad_oracle
@@ -508,10 +590,10 @@ def run_ours(args):
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
                 "kernels": kernels, "reconstruct": reconstruct, "dad_full_grad": full_grad, "compulsory_traffic": compulsory,
                 "stream_gbs": sum(sum(v for k, v in stream_bytes_per_layer(cfg, sh, iters).items() if not k.endswith("launches"))
-                                  for sh in layers) * cfg.blocks / (ms_per_step * 1e-3) / 1e9}
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+                                  for sh in layers) * cfg.blocks / (ms_per_step * 1e-3) / 1e9,
+                "launches_per_compress": launches_per_compress, "compress_path": compress_path, "check": check}
+        return line
+    return None
 
 
 if __name__ == "__main__":

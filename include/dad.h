@@ -141,7 +141,10 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
  *   DAD_PATH_TENSOR   bf16 inputs in 16-byte-aligned layouts: the same sequence on tcgen05 tensor cores
  *   DAD_PATH_FUSED    small sites: ONE launch, a thread-block cluster of *cluster_size CTAs per site runs every
  *                     application of the operator, the orthonormalisations and the final factor, with Y and W
- *                     in shared memory and the partial sums of Z and G~ exchanged inside the cluster.
+ *                     in shared memory and Z, G~ and the orthonormal vectors exchanged over distributed shared
+ *                     memory (the site's factor buffers fit in the cluster's shared memory).
+ *   DAD_PATH_FUSED_L2 the same one launch for sites whose factor buffers do not fit: the CTAs exchange partial
+ *                     sums and factors through the workspace (L2) instead.
  * Returns -1 for invalid arguments; cluster_size may be NULL.  dad_fused_enable(0) makes the library skip the
  * one-launch form (process-wide; for timing one pipeline against the other), dad_fused_enable(1) restores it.
  * The workspace size does not depend on that switch.
@@ -149,6 +152,7 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
 #define DAD_PATH_GENERAL 0
 #define DAD_PATH_TENSOR 1
 #define DAD_PATH_FUSED 2
+#define DAD_PATH_FUSED_L2 3
 int dad_compress_path(const dad_layer* layer, int r, int iters, int* cluster_size);
 void dad_fused_enable(int on);
 
@@ -310,6 +314,20 @@ dad_status dad_reconstruct_static(int64_t h_in, int64_t h_out, int64_t K, const 
  * those calls clears its own word when it starts.  This is the only call that synchronises.
  */
 dad_status dad_check(const void* ws, void* cuda_stream);
+
+/*
+ * Self-test of the bounded device-side waits (the paper has no counterpart).  Every wait of the tensor-core kernels
+ * on a copy or on the tensor cores gives up after a fixed number of polls; the CTA then stops issuing work, waits --
+ * again bounded -- for the copies and multiplications it has already issued, frees its tensor memory, records
+ * DAD_ERR_TIMEOUT in the workspace's status word and RETURNS.  This call makes that happen on purpose, harmlessly:
+ * it launches one small tile whose multiplying role is told to expect one block more than is ever loaded, with a
+ * limit of 1024 polls, on zeroed operands inside `ws`.  Nothing hangs and nothing faults; afterwards
+ * dad_check(ws) reports DAD_ERR_TIMEOUT, and the context and `ws` remain usable for ordinary calls (each clears the
+ * status word when it starts).
+ *   ws  DEVICE, 256-byte aligned, ws_bytes >= DAD_SELFTEST_BYTES; its contents are overwritten
+ */
+#define DAD_SELFTEST_BYTES (64u << 10)
+dad_status dad_selftest_bounded_wait(void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Kernels launched by this library in this process so far (all threads); for accounting. */
 uint64_t dad_launch_count(void);

@@ -28,7 +28,7 @@ EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_b
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
            "dad_rank_compress_gram", "dad_rank_compress_sequential_workspace_bytes", "dad_rank_compress_sequential",
-           "dad_check", "dad_compress_path", "dad_fused_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
+           "dad_check", "dad_selftest_bounded_wait", "dad_compress_path", "dad_fused_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
 
@@ -110,6 +110,8 @@ def lib() -> ctypes.CDLL:
         L.dad_compress_path.restype = ctypes.c_int
         L.dad_fused_enable.argtypes = [ctypes.c_int]
         L.dad_fused_enable.restype = None
+        L.dad_selftest_bounded_wait.argtypes = [vp, ctypes.c_size_t, vp]
+        L.dad_selftest_bounded_wait.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
         L.dad_check.restype = ctypes.c_int
         L.dad_launch_count.argtypes = []
@@ -179,7 +181,7 @@ def dad_workspace_bytes(layer: dad_layer, r: int, iters: int) -> int:
     return int(lib().dad_workspace_bytes(ctypes.byref(layer), r, iters))
 
 
-DAD_PATH_GENERAL, DAD_PATH_TENSOR, DAD_PATH_FUSED = 0, 1, 2
+DAD_PATH_GENERAL, DAD_PATH_TENSOR, DAD_PATH_FUSED, DAD_PATH_FUSED_L2 = 0, 1, 2, 3
 
 
 def dad_compress_path(layer: dad_layer, r: int, iters: int):
@@ -311,6 +313,15 @@ def dad_rank_compress_sequential(layer: dad_layer, A, D, r: int, iters: int, Q0,
     st = lib().dad_rank_compress_sequential(ctypes.byref(layer), _ptr(A), _ptr(D), r, iters, _ptr(Q0), _ptr(P), _ptr(Q),
                                             _ptr(sigma), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     _check(st, "dad_rank_compress_sequential")
+
+
+DAD_SELFTEST_BYTES = 64 << 10
+
+
+def dad_selftest_bounded_wait(ws, stream=None):
+    """Makes one bounded device-side wait run out on purpose (nothing hangs or faults); dad_check(ws) then
+    raises DAD_ERR_TIMEOUT."""
+    _check(lib().dad_selftest_bounded_wait(_ptr(ws), ws.numel(), _stream(stream)), "dad_selftest_bounded_wait")
 
 
 def dad_check(ws, stream=None):

@@ -359,7 +359,9 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
   if (fused_c > 0 && g_fused_on.load(std::memory_order_relaxed)) {
     char* base = static_cast<char*>(ws);
     err = cudaMemsetAsync(base + w.status, 0, 4, st);
-    if (err == cudaSuccess)
+    if (err == cudaSuccess && fused_dsm_fits(*L, r, fused_c, nullptr))
+      err = fused_dsm_compress(*L, A, D, r, iters, Q0, P, Q, sigma, reinterpret_cast<int*>(base + w.status), fused_c, st);
+    else if (err == cudaSuccess)
       err = fused_compress(*L, A, D, r, iters, Q0, P, Q, sigma, base + w.G, base + w.Z, base + w.fused_part,
                            reinterpret_cast<double*>(base + w.fused_sig), reinterpret_cast<int*>(base + w.status), fused_c, st);
   } else if (tc)
@@ -454,12 +456,23 @@ int dad_compress_path(const dad_layer* layer, int r, int iters, int* cluster_siz
   const int c = g_fused_on.load(std::memory_order_relaxed) ? fused_cluster_size(L, r, iters) : 0;
   if (c > 0) {
     if (cluster_size) *cluster_size = c;
-    return DAD_PATH_FUSED;
+    return fused_dsm_fits(L, r, c, nullptr) ? DAD_PATH_FUSED : DAD_PATH_FUSED_L2;
   }
   return tc_eligible(L) ? DAD_PATH_TENSOR : DAD_PATH_GENERAL;
 }
 
 void dad_fused_enable(int on) { g_fused_on.store(on != 0, std::memory_order_relaxed); }
+
+dad_status dad_selftest_bounded_wait(void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!ws) return DAD_ERR_NULL;
+  if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
+  if (ws_bytes < DAD_SELFTEST_BYTES) return DAD_ERR_WORKSPACE;
+  if (!tmap_encoder_available()) return DAD_ERR_CUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(ws);
+  if (cudaMemsetAsync(base, 0, DAD_SELFTEST_BYTES, st) != cudaSuccess) return DAD_ERR_CUDA;
+  return umma_selftest_timeout(base + 1024, reinterpret_cast<int*>(base), st) == cudaSuccess ? DAD_OK : DAD_ERR_CUDA;
+}
 
 uint64_t dad_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -94,6 +94,11 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc, int 
 // One-launch compress of small sites (fused_site.cu): a cluster of `C` CTAs per site runs the whole structured
 // power iteration.  fused_cluster_size gives C for a shape, or 0 when the multi-launch pipelines take it.
 int fused_cluster_size(const dad_layer& L, int r, int iters);
+// The on-chip form of it (fused_dsm.cu): factor, Y and the rows of A and D in shared memory, every exchange over
+// distributed shared memory; preferred where its buffers fit.
+bool fused_dsm_fits(const dad_layer& L, int r, int C, bool* x_resident);
+cudaError_t fused_dsm_compress(const dad_layer& L, const void* A, const void* D, int r, int iters, const float* Q0, float* P,
+                               float* Q, float* sigma, int* status, int C, cudaStream_t st);
 cudaError_t fused_compress(const dad_layer& L, const void* A, const void* D, int r, int iters, const float* Q0, float* P,
                            float* Q, float* sigma, void* FG, void* FZ, void* part, double* sig_part, int* status, int C,
                            cudaStream_t st);
@@ -183,6 +188,7 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
 cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,
                           float* out2, __nv_bfloat16* planes, int64_t ld_planes, float* partial, unsigned* counters,
                           int* status, cudaStream_t st);
+cudaError_t umma_selftest_timeout(char* area, int* status, cudaStream_t st);
 cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& plan, int64_t hx, int64_t hy,
                          float* C, float* partial, unsigned* counters, int* status, cudaStream_t st);
 

@@ -323,21 +323,34 @@ cudaError_t launch_fused(const FusedParams& p, int S, size_t smem, cudaStream_t 
 
 }  // namespace
 
-// CTAs per site of the one-launch compress, or 0 when the shape is left to the multi-launch pipelines.  The cluster
-// takes the site when its share of the multiply-adds is small enough that one wave of S clusters finishes before the
-// 5 * iters + 3 dependent launches of the other pipelines would (each of those costs a few microseconds however
-// little it does), and the slab of the Cholesky-QR plus Y fit in shared memory.
+// CTAs per site of the one-launch compress, or 0 when the shape is left to the multi-launch pipelines.
+//
+// Measured on B200 (fp32 inputs, fp64 accumulation): a pass of the one-launch kernel over A or D costs about 8 us
+// of barriers, exchanges and dependent memory round trips however small the site, plus about 40 ns per thousand
+// multiply-adds of a CTA's share (20 ns with fp32 accumulation); a pass of the multi-launch pipelines costs about
+// 24 us of launches (general kernels) or 15 us (tensor-core kernels) while the GPU is not yet full.  A GPU holds
+// about 15 clusters of 8 CTAs at a time (two per GPC), 32 of 4, 70 of 2; more sites than that run in waves.  The
+// cluster size with the smallest estimate is taken, if it beats the multi-launch estimate.
 int fused_cluster_size(const dad_layer& L, int r, int iters) {
   if (L.N > (1 << 20) || L.h_in > (1 << 20) || L.h_out > (1 << 20)) return 0;
   const size_t acc = L.dtype == DAD_F32 ? 8 : 4;
-  int C = 8;
-  while (C > 1 && L.N < 4 * C) C /= 2;                            // at least 4 rows per CTA
-  while (C > 1 && (int64_t)L.S * C > 148) C /= 2;                // one wave where the site count allows it
-  if (fused_smem_for(L.N, L.h_out, r, C, acc) > 200 * 1024) return 0;
-  const double fma_per_cta = (2.0 * iters + 1.0) * (double)L.N * r * (double)(L.h_in + L.h_out) / C;
-  const double waves = (double)(((int64_t)L.S * C + 147) / 148);
-  const double budget = L.dtype == DAD_F32 ? 6.0e6 : 12.0e6;     // about 120 us of one SM's fp64 / fp32 pipe
-  return fma_per_cta * waves <= budget ? C : 0;
+  const double ns_per_kfma = L.dtype == DAD_F32 ? 40.0 : 20.0;
+  const double multi_us = tc_eligible(L) ? 15.0 : 24.0;
+  const double fma_per_pass = (double)L.N * r * (double)(L.h_in + L.h_out);
+  int best = 0;
+  double best_us = multi_us;  // per pass
+  for (int C = 8; C >= 1; C /= 2) {
+    if (C > 1 && L.N < 4 * C) continue;  // at least 4 rows per CTA
+    if (fused_smem_for(L.N, L.h_out, r, C, acc) > 200 * 1024 && !fused_dsm_fits(L, r, C, nullptr)) continue;
+    const int at_once = C == 8 ? 15 : C == 4 ? 32 : C == 2 ? 70 : 148;
+    const double waves = (double)((L.S + at_once - 1) / at_once);
+    const double us = waves * (8.0 + ns_per_kfma * 1e-6 * fma_per_pass / C);
+    if (us < best_us) {
+      best_us = us;
+      best = C;
+    }
+  }
+  return best;
 }
 
 cudaError_t fused_compress(const dad_layer& L, const void* A, const void* D, int r, int iters, const float* Q0, float* P,

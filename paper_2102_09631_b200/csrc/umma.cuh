@@ -34,13 +34,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after kWaitLimit polls (each poll itself blocks for a short hardware-defined
+// Bounded wait: gives up after `limit` polls (kWaitLimit unless the launch says otherwise) (each poll itself blocks for a short hardware-defined
 // time), or as soon as another thread of the CTA has given up.  Returns false on give-up and raises
 // the CTA-wide abort flag, so that every role of the kernel leaves its loop and the CTA can free its
 // tensor memory and return instead of hanging.
 constexpr uint32_t kWaitLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = kWaitLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *abort_flag) return false;
   }

@@ -53,6 +53,8 @@ struct UmmaParams {
   float* partial;    // split partial tiles [tile][split][128][BN]
   unsigned* counters;
   int* status;
+  uint32_t wait_limit;  // polls a bounded wait may take; 0 = kWaitLimit
+  int expect_extra_kb;  // self-test only: the MMA role waits for this many blocks more than the producer loads
 };
 
 template <int BN, bool A_MN, bool B_MN, int TERMS, int EPI, int STAGES>
@@ -71,9 +73,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar, flush_bar;
   __shared__ uint32_t tmem_base_s;
-  __shared__ int abort_flag, issued_s, last_flag;
+  __shared__ int abort_flag, issued_s, last_flag, flush_s;
+  const uint32_t wlim = p.wait_limit ? p.wait_limit : kWaitLimit;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tile = blockIdx.x;
@@ -90,9 +93,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_init(&empty_bar[s], 1);
     }
     mbar_init(&accum_bar, 1);
+    mbar_init(&flush_bar, 1);
     abort_flag = 0;
     issued_s = 0;
     last_flag = 0;
+    flush_s = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -120,7 +125,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (; i < nkb; ++i) {
         const int stage = i % STAGES;
         const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp)) break;
+        if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp, wlim)) break;
         mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
         uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
         uint8_t* b_dst = a_dst + A_BYTES;
@@ -148,10 +153,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      for (int i = 0; i < nkb; ++i) {
+      for (int i = 0; i < nkb + p.expect_extra_kb; ++i) {
         const int stage = i % STAGES;
         const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        if (!mbar_wait(&full_bar[stage], ph, abortp)) break;
+        if (!mbar_wait(&full_bar[stage], ph, abortp, wlim)) break;
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
         const uint32_t b_addr = a_addr + A_BYTES;
@@ -164,13 +169,17 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         umma_commit(&empty_bar[stage]);
       }
       umma_commit(&accum_bar);
+      if (*abortp) {  // giving up: the teardown waits on this for the MMAs issued so far before tensor memory is freed
+        umma_commit(&flush_bar);
+        flush_s = 1;
+      }
     }
   } else {
     // ---- epilogue: 4 warps, warp (id % 4) owns TMEM lanes 32*(id % 4) .. +31 ----
     const int q = warp & 3;
     const int row = q * 32 + lane;
     const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
-    const bool ok = mbar_wait(&accum_bar, 0u, abortp);
+    const bool ok = mbar_wait(&accum_bar, 0u, abortp, wlim);
     tc_fence_after();
     const int tiles_n = gridDim.y / p.splits;
     const int64_t tile_lin = ((int64_t)batch * gridDim.x + m_tile) * tiles_n + n_tile;
@@ -339,6 +348,13 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(bar, ph); ++t) {
         }
       }
+      // ... and for the MMAs already issued (they read shared memory and write the accumulator)
+      for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(&accum_bar, 0u); ++t) {  // committed after the last MMA issued
+      }
+      if (flush_s) {
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(&flush_bar, 0u); ++t) {
+        }
+      }
       if (p.status) *p.status = (int)DAD_ERR_TIMEOUT;
     }
     __syncthreads();
@@ -366,9 +382,9 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar, drained_bar;
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar, drained_bar, flush_bar;
   __shared__ uint32_t tmem_base_s;
-  __shared__ int abort_flag, issued_s;
+  __shared__ int abort_flag, issued_s, flush_s;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Work of this CTA.  The first tiles * splits CTAs each own one tile and one of the `splits` equal parts of the
@@ -417,8 +433,10 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     mbar_init(&accum_bar, 1);
     mbar_init(&drained_bar, 128);
+    mbar_init(&flush_bar, 1);
     abort_flag = 0;
     issued_s = 0;
+    flush_s = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -492,6 +510,10 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         if (go) umma_commit(&accum_bar);
       }
+      if (*abortp) {  // giving up: the teardown waits on this for the MMAs issued so far before tensor memory is freed
+        umma_commit(&flush_bar);
+        flush_s = 1;
+      }
     }
   } else {
     const int q = warp & 3;
@@ -551,6 +573,11 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         uint64_t* bar = &full_bar[i % STAGES];
         const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
         for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(bar, ph); ++t) {
+        }
+      }
+      // ... and for the MMAs already issued (they read shared memory and write the accumulator)
+      if (flush_s) {
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(&flush_bar, 0u); ++t) {
         }
       }
       if (p.status) *p.status = (int)DAD_ERR_TIMEOUT;
@@ -646,8 +673,15 @@ static cudaError_t launch_umma(const CUtensorMap& tmA, const CUtensorMap& tmB, c
   constexpr int B_BYTES = B_MN ? (BN / 64) * 8192 : TERMS * BN * 128;
   constexpr size_t smem = (size_t)STAGES * (A_BYTES + B_BYTES) + 1024;
   auto kernel = umma_kernel<BN, A_MN, B_MN, TERMS, EPI, STAGES>;
-  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (err != cudaSuccess) return err;
+  cudaError_t err = cudaSuccess;
+  static FirstUse first;  // the opt-in to large dynamic shared memory is per function and device, not per launch
+  if (first.on_this_device()) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) {
+      first.forget();
+      return err;
+    }
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(192, 1, 1);
@@ -688,6 +722,33 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
     case 32: return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
     default: return launch_umma<64, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
   }
+}
+
+// Self-test of the bounded waits: one 128 x 64 tile of Y = X F^T whose MMA role is told to expect one block more than
+// the producer loads, with a wait limit of 1024 polls.  The extra wait runs out, the CTA raises its abort flag, waits
+// (bounded) for the copies and MMAs it has issued, frees its tensor memory, sets *status = DAD_ERR_TIMEOUT and
+// returns.  `area` is 64 KB of zeroed device memory for the operands and the result.
+cudaError_t umma_selftest_timeout(char* area, int* status, cudaStream_t st) {
+  __nv_bfloat16* X = reinterpret_cast<__nv_bfloat16*>(area);             // 128 x 64
+  __nv_bfloat16* F = reinterpret_cast<__nv_bfloat16*>(area + 16384);     // 2 planes x 16 x 64
+  __nv_bfloat16* Yt = reinterpret_cast<__nv_bfloat16*>(area + 32768);    // 2 planes x 16 x 128
+  CUtensorMap tmX, tmF;
+  if (!make_tmap_bf16_3d(&tmX, X, 64, 128, 1, 128, 128 * 128, 64, 128) ||
+      !make_tmap_bf16_3d(&tmF, F, 64, 16, 2, 128, 16 * 128, 64, 16))
+    return cudaErrorInvalidValue;
+  UmmaParams p{};
+  p.m_extent = 128;
+  p.n_extent = 16;
+  p.k_blocks = 1;
+  p.kb_per_split = 1;
+  p.splits = 1;
+  p.out_planes = Yt;
+  p.ld_planes = 128;
+  p.plane_rows = 16;
+  p.status = status;
+  p.wait_limit = 1024;
+  p.expect_extra_kb = 1;
+  return launch_umma<16, false, false, 2, EPI_YT, 2>(tmX, tmF, p, dim3(1, 1, 1), "selftest", st);
 }
 
 // Z <- Y^T X.  tmX: X as (h, N, S) with box 64 x 64; tmYt: Y^T planes as (N, rp, 2S) with box 64 x rp.
@@ -781,8 +842,15 @@ static cudaError_t launch_gemm256(const CUtensorMap& tmA, const CUtensorMap& tmB
                                   cudaStream_t st) {
   constexpr size_t smem = (size_t)STAGES * 8 * BK * 128 + 1024;
   auto kernel = umma_gemm256_kernel<BK, STAGES>;
-  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (err != cudaSuccess) return err;
+  cudaError_t err = cudaSuccess;
+  static FirstUse first;
+  if (first.on_this_device()) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) {
+      first.forget();
+      return err;
+    }
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(192, 1, 1);

@@ -30,19 +30,68 @@ def rel(x, ref):
     return float(np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-300))
 
 
+GUARD_BYTES = 4096
+
+
+class Guarded:
+    """A device buffer with a band of 0xFF bytes (a NaN pattern for floats) before and after the part handed to the
+    library: whatever the library writes outside its buffer shows up as a changed guard byte."""
+
+    def __init__(self, nbytes, dev):
+        self.n = int(nbytes)
+        self.full = torch.full((self.n + 2 * GUARD_BYTES,), 0xFF, dtype=torch.uint8, device=dev)
+        self.inner = self.full[GUARD_BYTES:GUARD_BYTES + self.n]
+
+    def view(self, shape, dtype):
+        return self.inner.view(dtype).view(shape)
+
+    def intact(self):
+        lo, hi = self.full[:GUARD_BYTES], self.full[GUARD_BYTES + self.n:]
+        return bool((lo == 0xFF).all()) and bool((hi == 0xFF).all())
+
+
+def guard_plan(B, plan, dev):
+    """Moves every output and scratch buffer of a LayerPlan into guarded storage; returns the guards by name."""
+    guards = {}
+
+    def move(name, t):
+        g = Guarded(t.numel() * t.element_size(), dev)
+        guards[name] = g
+        return g.view(t.shape, t.dtype)
+
+    aliased = plan.Pcat.data_ptr() == plan.P.data_ptr()
+    plan.P, plan.Q, plan.sigma = move("P", plan.P), move("Q", plan.Q), move("sigma", plan.sigma)
+    if aliased:
+        L = plan.layer
+        plan.Pcat, plan.Qcat = plan.P.view(L.S * plan.r, L.h_in), plan.Q.view(L.S * plan.r, L.h_out)
+    else:
+        plan.Pcat, plan.Qcat = move("Pcat", plan.Pcat), move("Qcat", plan.Qcat)
+    plan.grads = move("grad", plan.grads)
+    plan.grad = plan.grads[0] if plan.groups == 1 else plan.grads
+    plan.ws = move("ws", plan.ws)
+    plan.ws[:256].zero_()        # the status words start out clear
+    return guards
+
+
 def run_gpu_layer(B, A, D, Q0, r, iters, math=None):
-    """compress -> gather -> reconstruct and full_grad on the GPU; returns host float64 arrays."""
+    """compress -> gather -> reconstruct and full_grad on the GPU; returns host float64 arrays.  Every buffer the
+    library writes sits between guard bands, which must come back untouched."""
     dev = torch.device("cuda:0")
     Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
     plan = B.LayerPlan(Ad, Dd, r, iters)
+    guards = guard_plan(B, plan, dev)
     if math is not None:
         plan.math = math
     plan.step(Ad, Dd, Q0d)
-    full = torch.empty_like(plan.grad)
+    gfull = Guarded(plan.grad.numel() * 4, dev)
+    guards["full"] = gfull
+    full = gfull.view(plan.grad.shape, torch.float32)
     tx_dad = B.bytes_array(plan.layer.S)
     B.dad_full_grad(plan.layer, Ad, Dd, full, tx_dad, plan.ws)
     B.dad_check(plan.ws)
     torch.cuda.synchronize()
+    for name, g in guards.items():
+        assert g.intact(), f"the library wrote outside its {name} buffer"
     f = lambda t: t.double().cpu().numpy()
     return dict(P=f(plan.P), Q=f(plan.Q), sigma=f(plan.sigma), Pcat=f(plan.Pcat), Qcat=f(plan.Qcat), grad=f(plan.grad),
                 full=f(full), tx_rank=list(plan.bytes_tx), tx_dad=list(tx_dad), layer=plan.layer)
@@ -89,7 +138,7 @@ def check_layer(oracle, B, A, D, Q0, r, iters, tol, ortho_tol=1e-4, compare_fact
     (1, 32, 784, 1024, 8, 3, torch.float32),      # the aggregator's stacks of a small layer as one site
     (3, 70, 264, 520, 40, 2, torch.float32),      # large rank (8 x 8 register blocks in the Cholesky-QR), ragged rows
     (5, 37, 50, 70, 7, 12, torch.float32),        # odd everything, many iterations
-    (2, 300, 256, 512, 16, 2, torch.bfloat16),    # bf16 inputs small enough for one cluster: fp32 accumulation
+    (2, 100, 128, 256, 8, 2, torch.bfloat16),     # bf16 inputs small enough for one cluster: fp32 accumulation
     (3, 100, 70, 50, 7, 2, torch.bfloat16),
 ])
 def test_one_launch_compress_matches_oracle_and_the_multi_launch_pipeline(oracle, B, S, N, h_in, h_out, r, iters, dtype):
@@ -101,7 +150,7 @@ def test_one_launch_compress_matches_oracle_and_the_multi_launch_pipeline(oracle
     A, D = wl.decaying_layer(S, N, h_in, h_out, seed, dtype)
     Q0 = wl.start_block(S, r, h_out, seed)
     path, C = B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)
-    assert path == B.DAD_PATH_FUSED and C >= 1
+    assert path in (B.DAD_PATH_FUSED, B.DAD_PATH_FUSED_L2) and C >= 1
     tol = TOL[dtype]
     g1, o = check_layer(oracle, B, A, D, Q0, r, iters, tol, ortho_tol=1e-3 if dtype == torch.bfloat16 else 1e-4)
     before = B.dad_launch_count()
@@ -109,7 +158,7 @@ def test_one_launch_compress_matches_oracle_and_the_multi_launch_pipeline(oracle
     assert np.array_equal(g1["P"], g2["P"]) and np.array_equal(g1["Q"], g2["Q"]) and np.array_equal(g1["sigma"], g2["sigma"])
     B.dad_fused_enable(False)
     try:
-        assert B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)[0] != B.DAD_PATH_FUSED
+        assert B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)[0] in (B.DAD_PATH_GENERAL, B.DAD_PATH_TENSOR)
         g3 = run_gpu_layer(B, A, D, Q0, r, iters)
     finally:
         B.dad_fused_enable(True)
@@ -337,6 +386,28 @@ def test_nan_input_is_reported_not_trapped(B):
     B.dad_check(plan.ws)
 
 
+def test_bounded_wait_runs_out_reports_timeout_and_leaves_the_context_usable(oracle, B):
+    """The give-up path of the tensor-core kernels, exercised without hanging or faulting anything: a small tile
+    whose multiplying role expects one block more than is loaded, with a limit of 1024 polls.  The wait runs out,
+    the CTA drains what it issued, frees its tensor memory and returns; the status word says DAD_ERR_TIMEOUT; an
+    ordinary call on the same workspace afterwards is clean and correct."""
+    dev = torch.device("cuda:0")
+    S, N, h_in, h_out, r, iters = 2, 300, 256, 512, 16, 2
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 5, torch.bfloat16)
+    Q0 = wl.start_block(S, r, h_out, 5)
+    Ad, Dd, Q0d = A.to(dev), D.to(dev), Q0.to(dev)
+    plan = B.LayerPlan(Ad, Dd, r, iters)
+    assert plan.ws.numel() >= B.DAD_SELFTEST_BYTES
+    for _ in range(2):
+        B.dad_selftest_bounded_wait(plan.ws)
+        with pytest.raises(B.DadError, match="TIMEOUT"):
+            B.dad_check(plan.ws)
+        plan.step(Ad, Dd, Q0d)
+        B.dad_check(plan.ws)                       # the status word was cleared by the call; nothing else is reported
+        o = oracle.rank_dad_layer(A, D, Q0, iters)
+        assert rel(plan.grad.double().cpu().numpy(), o["grad"]) <= 1e-4
+
+
 def test_reconstruct_and_full_grad_at_full_size_on_sampled_rows(oracle, B):
     """Largest shapes of the GPT-2-medium configuration; the oracle computes sampled output rows."""
     dev = torch.device("cuda:0")
@@ -377,10 +448,60 @@ def test_compress_at_full_size_on_sampled_sites(oracle, B):
     Po, Qo, _ = oracle.spi_block(A[sites].cpu(), D[sites].cpu(), Q0[sites].cpu(), cfg.iters)
     for i, s in enumerate(sites):
         got = plan.P[s].double().cpu().numpy().T @ plan.Q[s].double().cpu().numpy()
-        assert rel(got, Po[i].T @ Qo[i]) <= 2e-2
+        assert rel(got, Po[i].T @ Qo[i]) <= ACCURACY_BAR   # the contract says 2e-2; what is delivered is pinned too
         Qg = plan.Q[s].double().cpu().numpy()
         assert np.linalg.norm(Qg @ Qg.T - np.eye(cfg.r)) <= 1e-3
     assert list(plan.bytes_tx) == [oracle.bytes_rank(cfg.r, shape.h_in, shape.h_out)] * cfg.S
+
+
+ACCURACY_BAR = 1e-4   # delivered accuracy of the bf16 path on these workloads is a few 1e-6: losing a plane would show
+
+
+def full_size_case(oracle, B, cfg_index, shape, r, iters, groups, sites, whole_layer=None):
+    """One call exactly as the benchmark launches it (same-shape layers of `groups` blocks stacked as extra slices);
+    the oracle recomputes the sampled sites and, if asked, one whole layer's reconstructed gradient."""
+    dev = torch.device("cuda:0")
+    cfg = wl.CONFIGS[cfg_index]
+    S = cfg.S
+    A, D = wl.decaying_layer(S * groups, cfg.N, shape[0], shape[1], 7000 + cfg_index * 10 + r, torch.bfloat16, device=dev)
+    Q0 = wl.start_block(S * groups, r, shape[1], 7000 + r, dev)
+    plan = B.LayerPlan(A, D, r, iters, groups=groups)
+    guards = guard_plan(B, plan, dev)
+    grads = plan.step(A, D, Q0)
+    B.dad_check(plan.ws)
+    for name, g in guards.items():
+        assert g.intact(), f"the library wrote outside its {name} buffer"
+    Po, Qo, _ = oracle.spi_block(A[sites].cpu(), D[sites].cpu(), Q0[sites].cpu(), iters)
+    for i, s in enumerate(sites):
+        got = plan.P[s].double().cpu().numpy().T @ plan.Q[s].double().cpu().numpy()
+        err = rel(got, Po[i].T @ Qo[i])
+        assert err <= ACCURACY_BAR, (s, err)
+        Qg = plan.Q[s].double().cpu().numpy()
+        assert np.linalg.norm(Qg @ Qg.T - np.eye(r)) <= 1e-3
+    assert list(plan.bytes_tx) == [oracle.bytes_rank(r, shape[0], shape[1])] * (S * groups)
+    if whole_layer is not None:
+        sl = slice(whole_layer * S, (whole_layer + 1) * S)
+        o = oracle.rank_dad_layer(A[sl].cpu(), D[sl].cpu(), Q0[sl].cpu(), iters)
+        g = grads[whole_layer] if groups > 1 else grads
+        err = rel(g.double().cpu().numpy(), o["grad"])
+        assert err <= ACCURACY_BAR, err
+
+
+def test_vit_b_configuration_at_its_own_size(oracle, B):
+    """Configuration 4 as the benchmark launches it: N = 6304 rows per site (49 row tiles of 128 and a 32-row
+    remainder), S = 8, r = 16, three iterations -- the attention projections of a block stacked in one call
+    (768 CTAs in the column products: their five-stage form), and one 768 -> 3072 layer."""
+    cfg = wl.CONFIGS[4]
+    assert (cfg.N, cfg.S, cfg.r) == (6304, 8, 16)
+    full_size_case(oracle, B, 4, (768, 768), cfg.r, cfg.iters, groups=4, sites=[0, 29], whole_layer=2)
+    full_size_case(oracle, B, 4, (768, 3072), cfg.r, cfg.iters, groups=1, sites=[3, 7])
+
+
+@pytest.mark.parametrize("shape,r,iters,groups", [((4096, 1024), 16, 3, 1),     # the down projection at full size
+                                                  ((1024, 1024), 4, 1, 16),     # the sweep's smallest rank, stacked call
+                                                  ((1024, 4096), 4, 3, 4)])
+def test_gpt2_medium_configuration_remaining_shapes_at_full_size(oracle, B, shape, r, iters, groups):
+    full_size_case(oracle, B, 5, shape, r, iters, groups, sites=[1, 16 * groups - 1])
 
 
 @pytest.mark.parametrize("r,iters", [(16, 3), (64, 1)])
@@ -404,13 +525,13 @@ def test_stacked_call_at_the_benchmarks_launch_shape(oracle, B, r, iters):
     Po, Qo, _ = oracle.spi_block(A[sites].cpu(), D[sites].cpu(), Q0[sites].cpu(), iters)
     for i, s in enumerate(sites):
         got = plan.P[s].double().cpu().numpy().T @ plan.Q[s].double().cpu().numpy()
-        assert rel(got, Po[i].T @ Qo[i]) <= 2e-2
+        assert rel(got, Po[i].T @ Qo[i]) <= ACCURACY_BAR
         Qg = plan.Q[s].double().cpu().numpy()
         assert np.linalg.norm(Qg @ Qg.T - np.eye(r)) <= 1e-3
     g = 6                                   # one whole layer of the stack: its 16 sites and its gradient
     sl = slice(g * S, (g + 1) * S)
     o = oracle.rank_dad_layer(A[sl].cpu(), D[sl].cpu(), Q0[sl].cpu(), iters)
-    assert rel(grads[g].double().cpu().numpy(), o["grad"]) <= 2e-2
+    assert rel(grads[g].double().cpu().numpy(), o["grad"]) <= ACCURACY_BAR
     assert list(plan.bytes_tx)[sl] == [int(x) for x in o["bytes_tx"]]
 
 
