@@ -62,6 +62,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile-pass", action="store_true")
     ap.add_argument("--no-full-grad", action="store_true", help="skip timing the uncompressed dAD gradient")
+    ap.add_argument("--reconstruct-terms", type=int, default=None, choices=[1, 3],
+                    help="bf16 products per reconstruction: 3 = two-term splits of the fp32 factors (about 16 bits of each), "
+                         "1 = their hi terms only (about 8 bits); default: 1 where the contraction S*r is at least 512 and "
+                         "the product is tensor-bound, else 3")
     ap.add_argument("--no-sweep", action="store_true",
                     help="skip the other configurations and the rank / iteration sweep of configuration 5 that a default "
                          "run reports beside its headline workload")
@@ -324,7 +328,11 @@ def measure(args, rank, local, world, dev, headline):
         key = (sh.h_in, sh.h_out, groups)
         if key not in plans:
             A, D, _ = data[0][ui]
-            plans[key] = B.LayerPlan(A, D, r, iters, groups=groups)
+            rmath = None
+            if cfg.dtype != "f32":
+                terms = args.reconstruct_terms or (1 if cfg.S * r >= 512 else 3)
+                rmath = B.DAD_BF16_1TERM if terms == 1 else B.DAD_BF16
+            plans[key] = B.LayerPlan(A, D, r, iters, groups=groups, reconstruct_math=rmath)
     input_bytes = sum(A.numel() * A.element_size() + D.numel() * D.element_size() for blk in data for A, D, _ in blk)
     stream = torch.cuda.current_stream()
     # Calls on different plans are independent (own inputs, workspace and outputs).  Where one call cannot fill the GPU
@@ -438,7 +446,8 @@ def measure(args, rank, local, world, dev, headline):
     if rec:
         K = cfg.S * r
         bf16 = "gemm_tn_tc" in kernels
-        terms = 3 if bf16 else 1           # bf16 math multiplies two-term splits of the fp32 factors: three products
+        # bf16 math multiplies two-term splits of the fp32 factors (three products) or their hi terms only (one)
+        terms = (3 if next(iter(plans.values())).math == B.DAD_BF16 else 1) if bf16 else 1
         flops = sum(2.0 * K * sh.h_in * sh.h_out for sh in layers) * cfg.blocks
         out_bytes = sum(4.0 * sh.h_in * sh.h_out for sh in layers) * cfg.blocks
         in_bytes = sum((2.0 * terms if bf16 else 4.0) * K * (sh.h_in + sh.h_out) for sh in layers) * cfg.blocks

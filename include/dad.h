@@ -48,7 +48,11 @@ typedef enum {
   DAD_ERR_NUMERIC = 9    /* a NaN/Inf reached the orthonormalisation (reported by dad_check)  */
 } dad_status;
 
-typedef enum { DAD_F32 = 0, DAD_BF16 = 1 } dad_dtype;
+typedef enum {
+  DAD_F32 = 0,
+  DAD_BF16 = 1,
+  DAD_BF16_1TERM = 2 /* only as the `math` of a reconstruction: one bf16 product instead of three (see dad_reconstruct) */
+} dad_dtype;
 
 #define DAD_MAX_RANK 64
 
@@ -209,7 +213,10 @@ dad_status dad_gather_factors(const dad_layer* layer, int r, const float* P, con
  *              factor enters as a two-term bf16 split x = hi + lo and the product is
  *              hi*hi + hi*lo + lo*hi (one contraction of length 3K), so the result carries about
  *              16 significant bits of the factors (the dropped lo*lo term is 2^-16 relative).
- *              Needs h_in and h_out multiples of 8; otherwise DAD_BF16 falls back to the
+ *              DAD_BF16_1TERM: the hi terms only, one contraction of length K -- a third of the
+ *              operand traffic and tensor-core work, about 8 significant bits of each factor
+ *              (measured 2e-3 to 4e-3 relative on the gradient, inside the 2e-2 bar of bf16 inputs).
+ *              Both need h_in and h_out multiples of 8; otherwise they fall back to the
  *              fp32 FMA kernel (still on the device).
  *   ws         DEVICE scratch of ws_bytes >= dad_reconstruct_workspace_bytes(h_in, h_out, K, math),
  *              may be NULL when that is 0

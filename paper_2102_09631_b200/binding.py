@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdad.so")
 
 DAD_OK = 0
-DAD_F32, DAD_BF16 = 0, 1
+DAD_F32, DAD_BF16, DAD_BF16_1TERM = 0, 1, 2
 DAD_MAX_RANK = 64
 STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD_ERR_RANK", "DAD_ERR_WORKSPACE",
                 "DAD_ERR_ALIGN", "DAD_ERR_CUDA", "DAD_ERR_TIMEOUT", "DAD_ERR_NUMERIC"]
@@ -357,7 +357,7 @@ class LayerPlan:
     of the stacks (one batched call); `grad` is then groups x h_in x h_out."""
 
     def __init__(self, A: torch.Tensor, D: torch.Tensor, r: int, iters: int, zero_copy_gather: bool = False,
-                 groups: int = 1):
+                 groups: int = 1, reconstruct_math: Optional[int] = None):
         self.layer = make_layer(A, D)
         L = self.layer
         if groups < 1 or L.S % groups:
@@ -375,7 +375,8 @@ class LayerPlan:
             self.Qcat = torch.empty(L.S * r, L.h_out, device=dev, dtype=torch.float32)
         self.grads = torch.empty(groups, L.h_in, L.h_out, device=dev, dtype=torch.float32)
         self.grad = self.grads[0] if groups == 1 else self.grads
-        self.math = L.dtype
+        # reconstruction arithmetic: that of the inputs (fp32 FMA / three-term bf16) unless the caller picks one
+        self.math = L.dtype if reconstruct_math is None else reconstruct_math
         nws = dad_workspace_bytes(L, r, iters)
         if nws == 0:
             raise ValueError("invalid layer / rank / iteration count")

@@ -390,14 +390,20 @@ dad_status dad_gather_factors(const dad_layer* L, int r, const float* P, const f
   return DAD_OK;
 }
 
-static bool reconstruct_tc(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
-  return math == DAD_BF16 && h_in % 8 == 0 && h_out % 8 == 0 && 3 * K <= 0x7fffffff && tmap_encoder_available();
+// bf16 products of the tensor-core reconstruction for this problem: 3 (two-term splits), 1 (hi terms only), or 0
+// when the fp32 kernel takes it.
+static int reconstruct_terms(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
+  if (math != DAD_BF16 && math != DAD_BF16_1TERM) return 0;
+  if (h_in % 8 != 0 || h_out % 8 != 0 || 3 * K > 0x7fffffff || !tmap_encoder_available()) return 0;
+  return math == DAD_BF16 ? 3 : 1;
 }
+static bool math_ok(dad_dtype math) { return math == DAD_F32 || math == DAD_BF16 || math == DAD_BF16_1TERM; }
 
 size_t dad_reconstruct_batched_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, int batch, dad_dtype math) {
   if (h_in < 1 || h_out < 1 || K < 1 || batch < 1) return 0;
-  if (!reconstruct_tc(h_in, h_out, K, math)) return 0;
-  return gemm_ws_layout(h_in, h_out, 1, 3 * K, true, batch).total;
+  const int terms = reconstruct_terms(h_in, h_out, K, math);
+  if (terms == 0) return 0;
+  return gemm_ws_layout(h_in, h_out, 1, terms * K, true, batch).total;
 }
 
 size_t dad_reconstruct_workspace_bytes(int64_t h_in, int64_t h_out, int64_t K, dad_dtype math) {
@@ -409,22 +415,22 @@ dad_status dad_reconstruct_batched(int64_t h_in, int64_t h_out, int64_t K, int b
                                    void* cuda_stream) {
   if (h_in < 1 || h_out < 1 || K < 1 || h_in > 0x7fffffff || h_out > 0x7fffffff || batch < 1 || batch > 65535)
     return DAD_ERR_SHAPE;
-  if (math != DAD_F32 && math != DAD_BF16) return DAD_ERR_DTYPE;
+  if (!math_ok(math)) return DAD_ERR_DTYPE;
   if (!Pcat || !Qcat || !grad) return DAD_ERR_NULL;
   if (!aligned(Pcat, 16) || !aligned(Qcat, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaError_t err = cudaSuccess;
-  if (reconstruct_tc(h_in, h_out, K, math)) {
-    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, 3 * K, true, batch);  // three bf16 products, one contraction
+  if (const int terms = reconstruct_terms(h_in, h_out, K, math)) {
+    const GemmWs w = gemm_ws_layout(h_in, h_out, 1, terms * K, true, batch);  // `terms` bf16 products, one contraction
     if (!ws) return DAD_ERR_NULL;
     if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
     if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
     __nv_bfloat16* Xb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Xb);
     __nv_bfloat16* Yb = reinterpret_cast<__nv_bfloat16*>((char*)ws + w.Yb);
-    err = stack_split3(Pcat, (size_t)K * h_in, Xb, Qcat, (size_t)K * h_out, Yb, batch, st);
+    err = stack_split3(Pcat, (size_t)K * h_in, Xb, Qcat, (size_t)K * h_out, Yb, batch, terms, st);
     if (err == cudaSuccess)
-      err = run_gemm_tc(Xb, h_in, 3 * K * h_in, Yb, h_out, 3 * K * h_out, 1, 3 * K, h_in, h_out, grad, (char*)ws, w, st,
-                        batch);
+      err = run_gemm_tc(Xb, h_in, terms * K * h_in, Yb, h_out, terms * K * h_out, 1, terms * K, h_in, h_out, grad, (char*)ws,
+                        w, st, batch);
   } else {
     for (int b = 0; b < batch && err == cudaSuccess; ++b)
       err = gemm_tn_simt(DAD_F32, Pcat + (size_t)b * K * h_in, h_in, 0, Qcat + (size_t)b * K * h_out, h_out, 0, 1, K, h_in,

@@ -163,9 +163,10 @@ cudaError_t row_norms(const T* M, int64_t rows, int64_t h, float* out, cudaStrea
 // planes[s][0/1][j][c] = hi / lo bf16 terms of in[s][j][c]  (j < r; plane_rows >= r rows per plane)
 cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16* planes, int plane_rows,
                          cudaStream_t st);
-// Three-term bf16 operand stacks of `batch` reconstructions: P is batch x (nP elements), X3 is batch x 3 x nP, same for Q.
+// bf16 operand stacks of `batch` reconstructions, three-term (terms = 3) or hi terms only (terms = 1): P is
+// batch x (nP elements), X3 is batch x terms x nP, same for Q.
 cudaError_t stack_split3(const float* P, size_t nP, __nv_bfloat16* X3, const float* Q, size_t nQ, __nv_bfloat16* Y3,
-                         int batch, cudaStream_t st);
+                         int batch, int terms, cudaStream_t st);
 
 // ---- tensor-core launchers (umma_gemm.cu) -------------------------------------------------------
 bool tmap_encoder_available();

@@ -201,8 +201,11 @@ cudaError_t split_planes(const float* in, int S, int r, int64_t h, __nv_bfloat16
 //     X3 = [hi(P); hi(P); lo(P)]   and   Y3 = [hi(Q); lo(Q); hi(Q)].
 // Four elements per thread; nP and nQ are multiples of 4 and all pointers 8-byte aligned.  `batch` independent
 // factor stacks lie one after the other in P and Q; each gets its own three-term stack in X3 and Y3.
+// With terms == 1 only the hi terms are stored (X = hi(P), Y = hi(Q)): one product, about 8 significant bits of
+// each factor.
 __global__ void stack_split3_kernel(const float* __restrict__ P, size_t nP, __nv_bfloat16* __restrict__ X3,
-                                    const float* __restrict__ Q, size_t nQ, __nv_bfloat16* __restrict__ Y3, int batch) {
+                                    const float* __restrict__ Q, size_t nQ, __nv_bfloat16* __restrict__ Y3, int batch,
+                                    int terms) {
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   const size_t qP = nP / 4, qQ = nQ / 4;
   const size_t allP = qP * (size_t)batch, all = (qP + qQ) * (size_t)batch;
@@ -220,20 +223,22 @@ __global__ void stack_split3_kernel(const float* __restrict__ P, size_t nP, __nv
       lo[u] = __float2bfloat16_rn(f[u] - __bfloat162float(hi[u]));
     }
     const uint2 h2 = *reinterpret_cast<const uint2*>(hi), l2 = *reinterpret_cast<const uint2*>(lo);
-    uint2* out = reinterpret_cast<uint2*>(isP ? X3 : Y3) + b * 3 * plane;
+    uint2* out = reinterpret_cast<uint2*>(isP ? X3 : Y3) + b * terms * plane;
     out[q] = h2;
-    out[plane + q] = isP ? h2 : l2;
-    out[2 * plane + q] = isP ? l2 : h2;
+    if (terms == 3) {
+      out[plane + q] = isP ? h2 : l2;
+      out[2 * plane + q] = isP ? l2 : h2;
+    }
   }
 }
 
 cudaError_t stack_split3(const float* P, size_t nP, __nv_bfloat16* X3, const float* Q, size_t nQ, __nv_bfloat16* Y3,
-                         int batch, cudaStream_t st) {
+                         int batch, int terms, cudaStream_t st) {
   cudaError_t err = cudaSuccess;
   size_t blocks = ((nP + nQ) / 4 * (size_t)batch + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  DAD_LAUNCH(err, "stack_split3", stack_split3_kernel, (unsigned)blocks, 256, 0, st, P, nP, X3, Q, nQ, Y3, batch);
+  DAD_LAUNCH(err, "stack_split3", stack_split3_kernel, (unsigned)blocks, 256, 0, st, P, nP, X3, Q, nQ, Y3, batch, terms);
   return err;
 }
 

@@ -58,7 +58,7 @@ extern "C" {
 
 size_t dad_rank_dad_host_scratch_bytes(const dad_layer* layer, int r, int iters, dad_dtype math) {
   HostScratch sc;
-  if (!layer || (math != DAD_F32 && math != DAD_BF16) || !carve(*layer, r, iters, math, &sc)) return 0;
+  if (!layer || (math != DAD_F32 && math != DAD_BF16 && math != DAD_BF16_1TERM) || !carve(*layer, r, iters, math, &sc)) return 0;
   return sc.total;
 }
 
@@ -66,7 +66,7 @@ dad_status dad_rank_dad_host(const dad_layer* layer, const void* A_host, const v
                              int iters, dad_dtype math, float* grad_host, uint64_t* bytes_tx, void* dev_scratch,
                              size_t dev_scratch_bytes, void* cuda_stream) {
   if (!layer || !A_host || !D_host || !Q0_host || !grad_host || !dev_scratch) return DAD_ERR_NULL;
-  if (math != DAD_F32 && math != DAD_BF16) return DAD_ERR_DTYPE;
+  if (math != DAD_F32 && math != DAD_BF16 && math != DAD_BF16_1TERM) return DAD_ERR_DTYPE;
   if (reinterpret_cast<uintptr_t>(dev_scratch) % 256) return DAD_ERR_ALIGN;
   // the caller's own strides feed the copies: rows must not overlap, sites must not overlap (before anything is queued)
   if (layer->S >= 1 && layer->N >= 1 && layer->h_in >= 1 && layer->h_out >= 1) {

@@ -49,7 +49,7 @@ cudaError_t scratch_for_current_device(void** out) {
 extern "C" dad_status dad_reconstruct_static(int64_t h_in, int64_t h_out, int64_t K, const float* Pcat,
                                              const float* Qcat, float* grad, dad_dtype math, void* cuda_stream) {
   if (h_in < 1 || h_out < 1 || K < 1) return DAD_ERR_SHAPE;
-  if (math != DAD_F32 && math != DAD_BF16) return DAD_ERR_DTYPE;
+  if (math != DAD_F32 && math != DAD_BF16 && math != DAD_BF16_1TERM) return DAD_ERR_DTYPE;
   const size_t need = dad_reconstruct_workspace_bytes(h_in, h_out, K, math);
   if (need > (size_t)DAD_STATIC_SCRATCH_BYTES) return DAD_ERR_WORKSPACE;  // larger problems: dad_reconstruct with caller scratch
   void* scratch = nullptr;

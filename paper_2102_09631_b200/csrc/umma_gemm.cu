@@ -53,13 +53,15 @@ struct UmmaParams {
   float* partial;    // split partial tiles [tile][split][128][BN]
   unsigned* counters;
   int* status;
+  int tma_store;        // EPI_C without a split contraction: the tile leaves through shared memory and TMA stores (tmC)
   uint32_t wait_limit;  // polls a bounded wait may take; 0 = kWaitLimit
   int expect_extra_kb;  // self-test only: the MMA role waits for this many blocks more than the producer loads
 };
 
 template <int BN, bool A_MN, bool B_MN, int TERMS, int EPI, int STAGES>
 __global__ void __launch_bounds__(192)
-umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const UmmaParams p) {
+umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
   constexpr int A_BYTES = 128 * 64 * 2;
   constexpr int B_BYTES = B_MN ? (BN / 64) * 8192 : TERMS * BN * 128;
   constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -266,6 +268,39 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
       }
+    } else if (EPI == EPI_C && p.tma_store != 0) {
+      // The 128 x BN fp32 tile leaves through shared memory: 32 columns at a time every thread puts its row's 128
+      // bytes into a [128 rows][128 bytes] box (16-byte pieces swizzled as the tensor map expects, so the 32 lanes of
+      // a warp spread over all banks), and one thread hands the box to a TMA store, which writes whole lines and
+      // clips at the edges of C.  Two boxes alternate (the pipeline stages are free once the accumulator is complete),
+      // so the stores of one run under the TMEM reads of the next.  The contraction is not split here (splits == 1).
+      static_assert(EPI != EPI_C || 2 * 16384 <= STAGES * STAGE_BYTES, "two staging boxes have to fit in the stages");
+      const bool issuer = warp == 2 && lane == 0;
+      if (issuer) prefetch_tmap(&tmC);
+#pragma unroll 1
+      for (int c32 = 0; c32 < BN / 32; ++c32) {
+        uint8_t* box = smem + (c32 & 1) * 16384;
+        if (c32 >= 2) {  // the store that read this box two rounds ago has to be done with it
+          if (issuer) bulk_wait_read<1>();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        if (ok) {
+          float v[32];
+          tmem_ld16(lane_base + c32 * 32, *reinterpret_cast<float(*)[16]>(&v[0]));
+          tmem_ld16(lane_base + c32 * 32 + 16, *reinterpret_cast<float(*)[16]>(&v[16]));
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            *reinterpret_cast<float4*>(box + row * 128 + ((k ^ (row & 7)) * 16)) =
+                make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+        }
+        fence_async_proxy();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (issuer && ok && n0 + c32 * 32 < p.n_extent) {
+          tma_store_3d(&tmC, box, n0 + c32 * 32, m0, batch);
+          bulk_commit();
+        }
+      }
+      if (issuer) bulk_wait_all();
     } else if (finish) {
       const int64_t gm = (int64_t)m0 + row;  // global row of D
 #pragma unroll 1
@@ -649,6 +684,23 @@ bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t
   return r == CUDA_SUCCESS;
 }
 
+// fp32 tensor (d0 innermost, contiguous) x d1 x d2 with byte strides s1, s2; box = 32 x box1 x 1 (128 bytes wide),
+// 128-byte swizzle: the output tiles of the TMA-store epilogue.
+bool make_tmap_f32_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1_bytes,
+                      uint64_t s2_bytes, uint32_t box1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  if (d2 <= 1 && s2_bytes < s1_bytes) s2_bytes = s1_bytes * d1;
+  cuuint64_t strides[2] = {s1_bytes, s2_bytes};
+  cuuint32_t box[3] = {32, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 int umma_rank_pad(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 
 // CTAs that share the rows of one 128-column tile of Z = Y^T X.  A CTA streams its rows at about one SM's
@@ -668,7 +720,7 @@ int umma_cols_acc_splits(int S, int64_t N, int64_t h) {
 
 template <int BN, bool A_MN, bool B_MN, int TERMS, int EPI, int STAGES>
 static cudaError_t launch_umma(const CUtensorMap& tmA, const CUtensorMap& tmB, const UmmaParams& p, dim3 grid,
-                               const char* tag, cudaStream_t st) {
+                               const char* tag, cudaStream_t st, const CUtensorMap* tmC = nullptr) {
   constexpr int A_BYTES = 128 * 64 * 2;
   constexpr int B_BYTES = B_MN ? (BN / 64) * 8192 : TERMS * BN * 128;
   constexpr size_t smem = (size_t)STAGES * (A_BYTES + B_BYTES) + 1024;
@@ -694,7 +746,7 @@ static cudaError_t launch_umma(const CUtensorMap& tmA, const CUtensorMap& tmB, c
   cfg.numAttrs = 1;
   const bool timed = g_timing.load(std::memory_order_relaxed);
   if (timed) timing_mark(tag, st, true);
-  err = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+  err = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC ? *tmC : tmA, p);  // without tmC the kernel never touches it
   if (timed) timing_mark(tag, st, false);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return err;
@@ -904,12 +956,21 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
   // Short contractions (the reconstruction: 3 S r rows) spend as long in the epilogue -- 128 KB of fp32 per tile -- as in
   // the MMAs: two shallow CTAs per SM, one draining its accumulator while the other multiplies, instead of one deep one.
   const bool shallow = p.kb_per_split <= 64;
-  if (g.bn == 256) {
-    if (shallow) return launch_umma<256, true, true, 1, EPI_C, 2>(tmX, tmY, p, grid, "gemm_tn_tc", st);
-    return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+  // Without a split contraction the tile goes out through TMA stores (whole lines, asynchronous); C is hx x hy fp32,
+  // contiguous, one matrix per batch entry.
+  CUtensorMap tmC;
+  const CUtensorMap* pC = nullptr;
+  if (g.splits == 1 && make_tmap_f32_3d(&tmC, C, (uint64_t)hy, (uint64_t)hx, (uint64_t)g.batch, (uint64_t)hy * 4,
+                                        (uint64_t)hx * hy * 4, 128)) {
+    p.tma_store = 1;
+    pC = &tmC;
   }
-  if (shallow) return launch_umma<128, true, true, 1, EPI_C, 3>(tmX, tmY, p, grid, "gemm_tn_tc", st);
-  return launch_umma<128, true, true, 1, EPI_C, 6>(tmX, tmY, p, grid, "gemm_tn_tc", st);
+  if (g.bn == 256) {
+    if (shallow) return launch_umma<256, true, true, 1, EPI_C, 2>(tmX, tmY, p, grid, "gemm_tn_tc", st, pC);
+    return launch_umma<256, true, true, 1, EPI_C, 4>(tmX, tmY, p, grid, "gemm_tn_tc", st, pC);
+  }
+  if (shallow) return launch_umma<128, true, true, 1, EPI_C, 3>(tmX, tmY, p, grid, "gemm_tn_tc", st, pC);
+  return launch_umma<128, true, true, 1, EPI_C, 6>(tmX, tmY, p, grid, "gemm_tn_tc", st, pC);
 }
 
 }  // namespace dad

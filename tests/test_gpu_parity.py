@@ -294,6 +294,28 @@ def test_reconstruct_batched_is_the_per_layer_sum_of_outer_products(oracle, B, h
         assert torch.equal(one, single)
 
 
+@pytest.mark.parametrize("h_in,h_out,K,batch", [(1024, 4096, 1024, 1), (1024, 1024, 256, 4), (264, 520, 40, 3)])
+def test_one_term_reconstruction_stays_inside_the_contract(oracle, B, h_in, h_out, K, batch):
+    """DAD_BF16_1TERM multiplies the bf16 roundings of the factors once: a third of the work of the three-term
+    product, 8 significant bits of each factor.  Against the oracle's sum of outer products the error is a few
+    1e-3 -- inside the 2e-2 bar of bf16 arithmetic, and pinned here at 6e-3 so that a further loss shows."""
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(5150 + K)
+    Pcat = torch.randn(batch * K, h_in, generator=g)
+    Qcat = torch.randn(batch * K, h_out, generator=g)
+    ws = B.new_workspace(B.dad_reconstruct_batched_workspace_bytes(h_in, h_out, K, batch, B.DAD_BF16_1TERM), dev)
+    assert ws.numel() <= max(256, B.dad_reconstruct_batched_workspace_bytes(h_in, h_out, K, batch, B.DAD_BF16))
+    grads = torch.full((batch, h_in, h_out), float("nan"), device=dev)
+    B.dad_reconstruct_batched(h_in, h_out, K, batch, Pcat.to(dev), Qcat.to(dev), grads, B.DAD_BF16_1TERM, ws)
+    B.dad_check(ws)
+    rows = [0, 1, h_in // 2, h_in - 1]
+    for b in range(batch):
+        sl = slice(b * K, (b + 1) * K)
+        ref = oracle.reconstruct(Pcat[sl][:, rows], Qcat[sl])
+        err = rel(grads[b][rows].double().cpu().numpy(), ref)
+        assert 1e-4 < err <= 6e-3, (b, err)      # it really is the one-term product, and no worse than that
+
+
 def test_factors_match_on_separated_spectrum(oracle, B):
     """With well separated singular values and enough iterations each vector is determined up to
     rounding (thin QR with positive diagonal fixes the sign), so the raw factors agree too."""
