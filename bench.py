@@ -66,6 +66,10 @@ def parse_args():
                     help="bf16 products per reconstruction: 3 = two-term splits of the fp32 factors (about 16 bits of each), "
                          "1 = their hi terms only (about 8 bits); default: 1 where the contraction S*r is at least 512 and "
                          "the product is tensor-bound, else 3")
+    ap.add_argument("--shard-sites", action="store_true",
+                    help="strong scaling over the ranks: every layer's S sites are dealt over the GPUs, each rank compresses "
+                         "its own, one all-gather of the factors (NCCL) gives every rank the stacks of all sites, and every "
+                         "rank reconstructs locally")
     ap.add_argument("--no-sweep", action="store_true",
                     help="skip the other configurations and the rank / iteration sweep of configuration 5 that a default "
                          "run reports beside its headline workload")
@@ -237,6 +241,13 @@ def run_ours(args):
     multi.init("nccl", dev)
     dad_build.build()
     B.lib()
+    if args.shard_sites:
+        line = measure_sharded(args, rank, world, dev)
+        if rank == 0:
+            print(json.dumps(line))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     line = measure(args, rank, local, world, dev, headline=True)
     default_workload = (args.config == 5 and args.rank is None and args.iters is None and args.blocks is None
                         and not args.no_group and not args.cuda_graph and args.streams is None)
@@ -261,6 +272,100 @@ def run_ours(args):
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def measure_sharded(args, rank, world, dev):
+    """Sites sharded over the ranks (Algorithm 1 with one exchange): per layer, dad_rank_compress on this rank's
+    sites, an all-gather of the factors into this rank's own memory, dad_reconstruct on the stacks of all sites.
+    Total work is fixed as ranks are added (strong scaling).  Inputs: every site's (A, Delta) from its own seed,
+    whichever rank holds it."""
+    import torch
+    from paper_2102_09631_b200 import binding as B, multi, workloads as wl
+    cfg = wl.CONFIGS[args.config]
+    if args.blocks is not None:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, blocks=max(1, min(cfg.blocks, args.blocks)))
+    r = args.rank or cfg.r
+    iters = cfg.iters if args.iters is None else args.iters
+    stream = torch.cuda.current_stream()
+    units = []
+    for li, sh in enumerate(cfg.layers):
+        shard = multi.SiteShardedLayer(cfg.S, r, sh.h_in, sh.h_out)
+        mine = shard.sites
+        if not mine:
+            raise SystemExit(f"more ranks ({world}) than sites ({cfg.S}): nothing to do for rank {rank}")
+        As, Ds, Qs = [], [], []
+        for site in mine:                       # a site's data depends on the site, not on the rank that holds it
+            seed = wl.seed_for(cfg.index, li * 1000 + site)
+            gen = wl.gaussian_layer if cfg.index == 1 else wl.decaying_layer
+            a, d = gen(1, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
+            As.append(a)
+            Ds.append(d)
+            Qs.append(wl.start_block(1, r, sh.h_out, seed, dev))
+        A, D, Q0 = torch.cat(As), torch.cat(Ds), torch.cat(Qs)
+        plan = B.LayerPlan(A, D, r, iters, zero_copy_gather=True)
+        K = cfg.S * r
+        math = plan.math
+        grad = torch.empty(sh.h_in, sh.h_out, device=dev, dtype=torch.float32)
+        ws_rec = B.new_workspace(B.dad_reconstruct_workspace_bytes(sh.h_in, sh.h_out, K, math), dev)
+        units.append((sh, shard, plan, A, D, Q0, grad, ws_rec, math, K))
+    ex_events = []
+
+    def step(record):
+        for sh, shard, plan, A, D, Q0, grad, ws_rec, math, K in units:
+            for _ in range(sh.count * cfg.blocks):
+                def compress(sites):
+                    B.dad_rank_compress(plan.layer, A, D, r, iters, Q0, plan.P, plan.Q, plan.sigma, plan.ws, stream)
+                    return plan.P, plan.Q
+
+                def reconstruct(Pcat, Qcat):
+                    B.dad_reconstruct(sh.h_in, sh.h_out, K, Pcat.contiguous(), Qcat.contiguous(), grad, math, ws_rec, stream)
+                    return grad
+
+                def on_exchange(begin):
+                    if record:
+                        ev = torch.cuda.Event(enable_timing=True)
+                        ev.record(stream)
+                        ex_events.append(ev)
+
+                shard.step(compress, reconstruct, on_exchange)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            multi.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step(False)
+    for u in units:
+        B.dad_check(u[2].ws)
+    sync_all()
+    launches0 = B.dad_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(True)
+    ev1.record(stream)
+    sync_all()
+    ms = multi.max_over_ranks(ev0.elapsed_time(ev1), dev) / args.steps
+    ex_ms = sum(ex_events[i].elapsed_time(ex_events[i + 1]) for i in range(0, len(ex_events), 2)) / args.steps
+    n_layers = cfg.n_layers()
+    sent = sum(shard.sent_bytes * sh.count for sh, shard, *_ in units) * cfg.blocks
+    expect = sum(B.dad_bytes_rank(plan.layer, r) * len(shard.sites) * sh.count for sh, shard, plan, *_ in units) * cfg.blocks
+    all_sent = multi.gather_counts([sent])
+    return {"metric": METRIC, "value": n_layers / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(cfg, r, iters),
+                       "parallelism": f"sites sharded over {world} rank(s): {cfg.S} sites -> "
+                                      f"{[len(multi.shard_units(cfg.S, k, world)) for k in range(world)]} per rank; one "
+                                      "all-gather of the factors per layer, every rank reconstructs"},
+            "gpu_launches": B.dad_launch_count() - launches0,
+            "exchange": {"collective": "all_gather (nccl)" if world > 1 else "none (one rank)",
+                         "sent_bytes_per_step_by_rank": [c[0] for c in all_sent],
+                         "equals_sum_of_dad_bytes_rank": sent == expect,
+                         "ms_per_step_this_rank": ex_ms, "share_of_step": ex_ms / ms if ms > 0 else None}}
 
 
 def oracle_check(cfg, r, iters, plan, A, D, Q0, site=0):

@@ -91,3 +91,33 @@ def allgather_factors(P_local: torch.Tensor, Q_local: torch.Tensor, n_sites: int
     Qs = [parts[k][cap * r * h_in:cap * r * h_in + counts[k] * r * h_out].reshape(counts[k] * r, h_out)
           for k in range(world)]
     return torch.cat(Ps), torch.cat(Qs)
+
+
+class SiteShardedLayer:
+    """One linear layer whose S sites are dealt over the ranks (`shard_units`): rank k compresses its own sites,
+    one all-gather of the fp32 factors lands the stacks of ALL sites in every rank's own memory (Algorithm 1's
+    vertcat at the aggregator and its broadcast back, as a single exchange), and every rank reconstructs the same
+    gradient locally.  The arithmetic is supplied by the caller -- the library's calls on CUDA tensors over nccl, or
+    any stand-in on CPU tensors over gloo -- so that this exchange logic is the same code in both settings:
+
+        compress(site_indices) -> (P_local, Q_local)   S_local x r x h_in / h_out, this rank's sites in order
+        reconstruct(Pcat, Qcat) -> gradient             from the (S*r)-row stacks
+
+    `sent_bytes` is what this rank contributes to the exchange for one layer: r*(h_in+h_out)*4 per own site, the
+    rank-dAD transmission count of those sites."""
+
+    def __init__(self, n_sites: int, r: int, h_in: int, h_out: int):
+        rank, world = (dist.get_rank(), dist.get_world_size()) if (dist.is_available() and dist.is_initialized()) else (0, 1)
+        self.n_sites, self.r, self.h_in, self.h_out = n_sites, r, h_in, h_out
+        self.rank, self.world = rank, world
+        self.sites = shard_units(n_sites, rank, world)
+        self.sent_bytes = len(self.sites) * r * (h_in + h_out) * 4
+
+    def step(self, compress, reconstruct, on_exchange=None):
+        P_local, Q_local = compress(self.sites)
+        if on_exchange is not None:
+            on_exchange(True)
+        Pcat, Qcat = allgather_factors(P_local, Q_local, self.n_sites)
+        if on_exchange is not None:
+            on_exchange(False)
+        return reconstruct(Pcat, Qcat)

@@ -61,10 +61,26 @@ def _gather_worker(rank, world, port, out_dir):
     S, N, h_in, h_out, r, iters = 5, 12, 10, 9, 2, 2         # 5 sites over 2 ranks: 3 + 2
     A, D = wl.gaussian_layer(S, N, h_in, h_out, 321)
     Q0 = wl.start_block(S, r, h_out, 321)
-    mine = multi.shard_units(S, rank, world)
-    P, Q, _ = dad_oracle.spi_block(A[mine], D[mine], Q0[mine], iters)      # this rank compresses its own sites
-    Pcat, Qcat = multi.allgather_factors(torch.from_numpy(P), torch.from_numpy(Q), S)
-    grad = dad_oracle.reconstruct(Pcat.numpy(), Qcat.numpy())             # every rank reconstructs the same gradient
+    # the exchange logic the benchmark's --shard-sites mode runs (multi.SiteShardedLayer), here on CPU tensors over
+    # gloo with the oracle standing in for the library's compress and reconstruct
+    shard = multi.SiteShardedLayer(S, r, h_in, h_out)
+    mine = shard.sites
+    assert mine == multi.shard_units(S, rank, world)
+    stacks = {}
+
+    def compress(sites):
+        P, Q, _ = dad_oracle.spi_block(A[sites], D[sites], Q0[sites], iters)   # this rank compresses its own sites
+        return torch.from_numpy(P), torch.from_numpy(Q)
+
+    def reconstruct(Pc, Qc):
+        stacks["P"], stacks["Q"] = Pc, Qc
+        return dad_oracle.reconstruct(Pc.numpy(), Qc.numpy())                # every rank reconstructs the same gradient
+
+    marks = []
+    grad = shard.step(compress, reconstruct, on_exchange=marks.append)
+    assert marks == [True, False]
+    assert shard.sent_bytes == len(mine) * dad_oracle.bytes_rank(r, h_in, h_out)
+    Pcat, Qcat = stacks["P"], stacks["Q"]
     ref = dad_oracle.rank_dad_layer(A, D, Q0, iters)                       # all sites in one process
     ok = (np.array_equal(Pcat.numpy(), ref["Pcat"]) and np.array_equal(Qcat.numpy(), ref["Qcat"])
           and np.array_equal(grad, ref["grad"]))
