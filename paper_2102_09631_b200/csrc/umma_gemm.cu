@@ -53,6 +53,7 @@ struct UmmaParams {
   float* partial;    // split partial tiles [tile][split][128][BN]
   unsigned* counters;
   int* status;
+  int batch_count;      // persistent dense-product kernel: products in the launch (its grid is one-dimensional)
   int tma_store;        // EPI_C without a split contraction: the tile leaves through shared memory and TMA stores (tmC)
   uint32_t wait_limit;  // polls a bounded wait may take; 0 = kWaitLimit
   int expect_extra_kb;  // self-test only: the MMA role waits for this many blocks more than the producer loads
@@ -625,6 +626,209 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
 }
 
+// Dense product C = X^T Y for SHORT contractions (the reconstruction P^T Q of Algorithm 1, K = S r), persistent form:
+// one CTA per SM walks over 128 x 256 output tiles (all products of a batched call), with TWO accumulators in tensor
+// memory (2 x 256 columns), so that the tensor cores fill one while the epilogue drains the other.  With K of a few
+// hundred a tile's MMAs last about a microsecond and its 128 KB of fp32 output two or three: what bounds the product
+// is writing C, and per-tile CTAs spend as long starting, filling their pipeline and waiting for their last stores
+// as they spend on the tile.  Here the set-up happens once per SM, the stage ring runs on across tiles, and the
+// output leaves through two staging boxes and TMA stores (whole lines, clipped at the edges of C) that never block
+// the next tile.  Measured against the per-tile CTAs (two per SM) on 144 reconstructions of 1024 x 1024 ... 4096 per
+// step: 4 blocks per tile 0.453 against 0.466 ms, 12 blocks 0.725 against 0.703, 16 blocks 1.03 against 0.94 -- so it
+// takes the products of at most 8 blocks only.  (Staging the whole tile at once -- one proxy fence and two barriers
+// per tile instead of per 32 columns, with two pipeline stages -- was slower still: 0.507 ms.)  Roles, bounded waits and teardown as in umma_kernel; the contraction is never split.
+template <int STAGES>
+__global__ void __launch_bounds__(192)
+umma_gemm_persist_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
+  constexpr int BN = 256;
+  constexpr int A_BYTES = 2 * 8192, B_BYTES = 4 * 8192, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int BOX_BYTES = 128 * 128;  // [128 rows][32 fp32]
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t IDESC = instr_desc(128, BN, true, true);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* boxes = smem + (size_t)STAGES * STAGE_BYTES;
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2], flush_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag, issued_s, flush_s, epi_bad;
+  const uint32_t wlim = p.wait_limit ? p.wait_limit : kWaitLimit;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int per_product = p.tiles_m * p.tiles_n;
+  const int n_tiles = per_product * p.batch_count;
+  const int nkb = p.k_blocks;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 128);
+    }
+    mbar_init(&flush_bar, 1);
+    abort_flag = 0;
+    issued_s = 0;
+    flush_s = 0;
+    epi_bad = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_s, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  volatile int* abortp = &abort_flag;
+
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // tile t: product t / per_product; inside it m fastest, so that CTAs working side by side share a panel of Y
+  auto tile_at = [&](int t, int& m0, int& n0, int& bz) {
+    bz = t / per_product;
+    const int rem = t - bz * per_product;
+    n0 = (rem / p.tiles_m) * BN;
+    m0 = (rem % p.tiles_m) * 128;
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmA);
+      prefetch_tmap(&tmB);
+      int g = 0;
+      bool go = true;
+      for (int t = blockIdx.x; go && t < n_tiles; t += gridDim.x) {
+        int m0, n0, bz;
+        tile_at(t, m0, n0, bz);
+        for (int kb = 0; kb < nkb; ++kb, ++g) {
+          const int stage = g % STAGES;
+          const uint32_t ph = (uint32_t)(g / STAGES) & 1u;
+          if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp, wlim)) {
+            go = false;
+            break;
+          }
+          mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+          uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_BYTES;
+          const int kcoord = kb * 64;
+          tma_load_3d(a_dst, &tmA, &full_bar[stage], m0, kcoord, bz);
+          tma_load_3d(a_dst + 8192, &tmA, &full_bar[stage], m0 + 64, kcoord, bz);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tma_load_3d(b_dst + c * 8192, &tmB, &full_bar[stage], n0 + c * 64, kcoord, bz);
+          issued_s = g + 1;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int g = 0, it = 0;
+      bool go = true;
+      for (int t = blockIdx.x; go && t < n_tiles; t += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const uint32_t uses = (uint32_t)(it >> 1);
+        // the epilogue has read this accumulator's previous tile out (passes at once on its first use)
+        if (!mbar_wait(&acc_empty[buf], (uses & 1u) ^ 1u, abortp, wlim)) break;
+        tc_fence_after();
+        const uint32_t acc = tmem_base + (uint32_t)buf * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++g) {
+          const int stage = g % STAGES;
+          const uint32_t ph = (uint32_t)(g / STAGES) & 1u;
+          if (!mbar_wait(&full_bar[stage], ph, abortp, wlim)) {
+            go = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k16 = 0; k16 < 4; ++k16)
+            umma_bf16(acc, desc_mn_major(a_addr, k16), desc_mn_major(b_addr, k16), IDESC, (kb | k16) != 0 ? 1u : 0u);
+          umma_commit(&empty_bar[stage]);
+        }
+        if (go) umma_commit(&acc_full[buf]);
+      }
+      if (*abortp) {  // giving up: the teardown waits on this for the MMAs issued so far before tensor memory is freed
+        umma_commit(&flush_bar);
+        flush_s = 1;
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const bool issuer = warp == 2 && lane == 0;
+    if (issuer) prefetch_tmap(&tmC);
+    int it = 0, boxes_used = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+      int m0, n0, bz;
+      tile_at(t, m0, n0, bz);
+      const int buf = it & 1;
+      const uint32_t uses = (uint32_t)(it >> 1);
+      if (!mbar_wait(&acc_full[buf], uses & 1u, abortp, wlim)) epi_bad = 1;
+      asm volatile("bar.sync 1, 128;" ::: "memory");  // the four warps go on, or stop, together
+      if (*reinterpret_cast<volatile int*>(&epi_bad)) break;
+      tc_fence_after();
+      const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN;
+#pragma unroll 1
+      for (int c32 = 0; c32 < BN / 32; ++c32, ++boxes_used) {
+        uint8_t* box = boxes + (boxes_used & 1) * BOX_BYTES;
+        if (boxes_used >= 2) {  // the store that read this box two rounds ago has to be done with it
+          if (issuer) bulk_wait_read<1>();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        float v[32];
+        tmem_ld16(lane_base + c32 * 32, *reinterpret_cast<float(*)[16]>(&v[0]));
+        tmem_ld16(lane_base + c32 * 32 + 16, *reinterpret_cast<float(*)[16]>(&v[16]));
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          *reinterpret_cast<float4*>(box + row * 128 + ((k ^ (row & 7)) * 16)) =
+              make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+        fence_async_proxy();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (issuer) {
+          if (n0 + c32 * 32 < p.n_extent) tma_store_3d(&tmC, box, n0 + c32 * 32, m0, bz);
+          bulk_commit();  // (an empty group where the box lies beyond C, so that the count of groups stays in step)
+        }
+      }
+      // this thread's part of the accumulator is in shared memory: the tensor cores may overwrite it
+      tc_fence_before();
+      mbar_arrive(&acc_empty[buf]);
+    }
+    if (issuer) bulk_wait_all();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    if (threadIdx.x == 0) {
+      const int issued = issued_s;
+      const int first = issued > STAGES ? issued - STAGES : 0;
+      for (int i = first; i < issued; ++i) {
+        uint64_t* bar = &full_bar[i % STAGES];
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(bar, ph); ++t) {
+        }
+      }
+      if (flush_s) {
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(&flush_bar, 0u); ++t) {
+        }
+      }
+      if (p.status) *p.status = (int)DAD_ERR_TIMEOUT;
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+
 // C[m][n] = sum over splits, in split order, of the partial tiles umma_gemm256_kernel stored
 // ([tile][split][256][256] fp32): four columns per thread, the whole GPU instead of one CTA per tile.
 __global__ void __launch_bounds__(256)
@@ -673,15 +877,44 @@ bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t
                        uint64_t s2_bytes, uint32_t box0, uint32_t box1) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  cuuint64_t dims[3] = {d0, d1, d2};
   if (d2 <= 1 && s2_bytes < s1_bytes) s2_bytes = s1_bytes * d1;
+  // A map is a pure function of these nine numbers, and callers ask for the same few again and again (the planes
+  // of a workspace never move, a layer's inputs rarely do): the last encodings of this thread are kept.
+  struct Key {
+    const void* base;
+    uint64_t d0, d1, d2, s1, s2;
+    uint32_t b0, b1;
+    bool operator==(const Key& o) const {
+      return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && s1 == o.s1 && s2 == o.s2 && b0 == o.b0 && b1 == o.b1;
+    }
+  };
+  constexpr int kSlots = 64;
+  struct Slot {
+    Key key;
+    CUtensorMap map;
+    bool used;
+  };
+  static thread_local Slot cache[kSlots] = {};
+  static thread_local unsigned next = 0;
+  const Key key{base, d0, d1, d2, s1_bytes, s2_bytes, box0, box1};
+  for (int i = 0; i < kSlots; ++i)
+    if (cache[i].used && cache[i].key == key) {
+      *map = cache[i].map;
+      return true;
+    }
+  cuuint64_t dims[3] = {d0, d1, d2};
   cuuint64_t strides[2] = {s1_bytes, s2_bytes};
   cuuint32_t box[3] = {box0, box1, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  if (r != CUDA_SUCCESS) return false;
+  Slot& slot = cache[next++ % kSlots];
+  slot.key = key;
+  slot.map = *map;
+  slot.used = true;
+  return true;
 }
 
 // fp32 tensor (d0 innermost, contiguous) x d1 x d2 with byte strides s1, s2; box = 32 x box1 x 1 (128 bytes wide),
@@ -921,6 +1154,39 @@ static cudaError_t launch_gemm256(const CUtensorMap& tmA, const CUtensorMap& tmB
   return err;
 }
 
+template <int STAGES>
+static cudaError_t launch_gemm_persist(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                                       const UmmaParams& p, unsigned ctas, cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * (6 * 8192) + 2 * 128 * 128 + 1024;
+  auto kernel = umma_gemm_persist_kernel<STAGES>;
+  cudaError_t err = cudaSuccess;
+  static FirstUse first;
+  if (first.on_this_device()) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) {
+      first.forget();
+      return err;
+    }
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctas, 1, 1);
+  cfg.blockDim = dim3(192, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const bool timed = g_timing.load(std::memory_order_relaxed);
+  if (timed) timing_mark("gemm_tn_tc", st, true);
+  err = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
+  if (timed) timing_mark("gemm_tn_tc", st, false);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return err;
+}
+
+
 // C (hx x hy, fp32) <- sum over sites and rows of X^T Y.  tmX: (hx, N, S), tmY: (hy, N, S), boxes 64 x plan.bk.
 // With plan.batch > 1 (and S = 1) the third tensor dimension counts independent products instead: C is batch x hx x hy.
 cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& g, int64_t hx, int64_t hy,
@@ -964,6 +1230,13 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
                                         (uint64_t)hx * hy * 4, 128)) {
     p.tma_store = 1;
     pC = &tmC;
+  }
+  // Many 128 x 256 tiles of a short contraction over one site per product: the persistent kernel (one CTA per SM, two
+  // accumulators).  Its blocks are numbered per product, so a contraction over several sites keeps the per-tile CTAs.
+  const int64_t all_tiles = g.tiles * g.batch;
+  if (pC && g.bn == 256 && all_tiles >= 148 && p.k_blocks <= 8 && (g.batch > 1 || g.k_blocks == g.kb_per_site)) {
+    p.batch_count = g.batch;
+    return launch_gemm_persist<3>(tmX, tmY, tmC, p, 148u, st);
   }
   if (g.bn == 256) {
     if (shallow) return launch_umma<256, true, true, 1, EPI_C, 2>(tmX, tmY, p, grid, "gemm_tn_tc", st, pC);

@@ -271,7 +271,9 @@ def test_full_grad_with_remainder_ctas(oracle, B, h_in, h_out):
     assert rel(grads[0][rows].double().numpy(), ref) <= 1e-4
 
 
-@pytest.mark.parametrize("h_in,h_out,K,batch", [(1024, 1024, 256, 16), (264, 520, 40, 3), (70, 50, 12, 2)])
+@pytest.mark.parametrize("h_in,h_out,K,batch", [(1024, 1024, 256, 16), (264, 520, 40, 3), (70, 50, 12, 2),
+                                                (520, 5000, 40, 6),     # 600 tiles, ragged last tile row and column:
+                                                (2048, 4104, 72, 1)])   # the persistent kernel, batched and single
 def test_reconstruct_batched_is_the_per_layer_sum_of_outer_products(oracle, B, h_in, h_out, K, batch):
     """Algorithm 1's P^T Q step for several layers of one shape in one call: every entry against the oracle's
     sum of outer products over its own K rows of the stacks, and batch = 1 against dad_reconstruct bit for bit."""
