@@ -48,6 +48,9 @@ def parse_args():
                     help="distinct transformer blocks of input data kept in HBM and cycled through")
     ap.add_argument("--blocks", type=int, default=None,
                     help="run only this many of the network's blocks per step (profiling captures); default all")
+    ap.add_argument("--rows", type=int, default=None,
+                    help="rows per site instead of the configuration's N (reduced-size profiler captures of the same launch "
+                         "shapes: the CTA count of the streaming kernels does not depend on it once the rows are not split)")
     ap.add_argument("--group-blocks", type=int, default=4,
                     help="stack the same-shape layers of this many consecutive blocks into one call")
     ap.add_argument("--no-group", action="store_true",
@@ -250,6 +253,7 @@ def run_ours(args):
         return
     line = measure(args, rank, local, world, dev, headline=True)
     default_workload = (args.config == 5 and args.rank is None and args.iters is None and args.blocks is None
+                        and args.rows is None
                         and not args.no_group and not args.cuda_graph and args.streams is None)
     if default_workload and not args.no_sweep and world == 1:
         sweep = []
@@ -388,9 +392,12 @@ def measure(args, rank, local, world, dev, headline):
     from paper_2102_09631_b200 import binding as B, multi, workloads as wl
 
     cfg = wl.CONFIGS[args.config]
-    if args.blocks is not None:
+    if args.blocks is not None or args.rows is not None:
         import dataclasses
-        cfg = dataclasses.replace(cfg, blocks=max(1, min(cfg.blocks, args.blocks)))
+        if args.blocks is not None:
+            cfg = dataclasses.replace(cfg, blocks=max(1, min(cfg.blocks, args.blocks)))
+        if args.rows is not None:
+            cfg = dataclasses.replace(cfg, N=max(1, args.rows))
     r = args.rank or cfg.r
     iters = cfg.iters if args.iters is None else args.iters
     layers = expand_layers(cfg)

@@ -312,20 +312,21 @@ __device__ __noinline__ void dsm_cols_slice(const DsmCtx<TIn, TAcc>& cx, const T
         }
       }
       if (parts > 1) {
-        // `red` holds one value set per thread (kThreads x kVecBlock): the two columns of a thread take turns
+        // `red` holds one value set per thread (kVecBlock x kThreads, a thread's values kThreads apart so that a warp's
+        // stores fall into different banks): the two columns of a thread take turns
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           if (u > 0) __syncthreads();
           if (active) {
 #pragma unroll
-            for (int jj = 0; jj < kVecBlock; ++jj) cx.red[(part * cols + col) * kVecBlock + jj] = acc[u][jj];
+            for (int jj = 0; jj < kVecBlock; ++jj) cx.red[jj * kThreads + part * cols + col] = acc[u][jj];
           }
           __syncthreads();
           if (part == 0) {
 #pragma unroll 1
             for (int q = 1; q < parts; ++q)
 #pragma unroll
-              for (int jj = 0; jj < kVecBlock; ++jj) acc[u][jj] += cx.red[(q * cols + col) * kVecBlock + jj];
+              for (int jj = 0; jj < kVecBlock; ++jj) acc[u][jj] += cx.red[jj * kThreads + q * cols + col];
           }
         }
       }
