@@ -24,12 +24,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum divided by the algorithmic bytes of the same launch, from one ncu
-# capture of each kernel on the 1024-wide layers of this workload (536.9 MB per launch).  DRAM traffic of these
-# streaming kernels grows in proportion to the slices a launch covers, so the ratio carries over to the larger
-# launches timed here.  Set an entry to None when its kernel changes until the counters are taken again.
-# rows_dot_tc: recaptured after its epilogue change (1.040 / 1.038).  cols_acc_tc: its 2048-CTA launches now take a
-# two-stage form that has not been captured (1.043 for the five-stage one).
-DRAM_TRAFFIC_OVER_ALGORITHMIC = {"rows_dot_tc": 1.039, "cols_acc_tc": None}
+# capture of each kernel at this workload's launch shapes with 512 rows per site (268.4 MB per launch).  The
+# streamed operand and the Y^T planes grow with the rows, the factor planes do not; scaled to the 4096-row launches
+# timed here that gives the ratios below.  Set an entry to None when its kernel changes until the counters are taken
+# again.
+DRAM_TRAFFIC_OVER_ALGORITHMIC = {"rows_dot_tc": 1.039, "cols_acc_tc": 1.047}
 
 METRIC = "rank-dAD compress+reconstruct layers/s"
 UNIT = "layers/s"
