@@ -124,6 +124,42 @@ def test_bad_arguments_are_rejected_before_any_launch(B):
         assert len(lib.dad_status_string(code)) > 0
 
 
+def test_pipeline_query_and_diagnostics_validate_their_arguments(B):
+    lib = B.lib()
+    before = B.dad_launch_count()
+    E = {n: i for i, n in enumerate(B.STATUS_NAMES)}
+    c = ctypes.c_int(7)
+    # invalid layers / ranks give -1 and a cluster size of 0
+    assert lib.dad_compress_path(None, 4, 2, ctypes.byref(c)) == -1 and c.value == 0
+    assert lib.dad_compress_path(ctypes.byref(layer(B, N=0)), 4, 2, None) == -1
+    assert lib.dad_compress_path(ctypes.byref(layer(B)), 33, 2, None) == -1
+    assert lib.dad_compress_path(ctypes.byref(layer(B, dtype=2)), 4, 2, None) == -1    # DAD_BF16_1TERM is no storage type
+    # a small fp32 layer goes to a one-launch form; switching those off sends it to the general pipeline; the
+    # workspace size does not depend on the switch
+    L = layer(B)
+    n_on = B.dad_workspace_bytes(L, 4, 2)
+    path, C = B.dad_compress_path(L, 4, 2)
+    assert path in (B.DAD_PATH_FUSED, B.DAD_PATH_FUSED_L2) and 1 <= C <= 8 and L.N >= 4 * C
+    B.dad_fused_enable(False)
+    try:
+        assert B.dad_compress_path(L, 4, 2) == (B.DAD_PATH_GENERAL, 0)
+        assert B.dad_workspace_bytes(L, 4, 2) == n_on
+    finally:
+        B.dad_fused_enable(True)
+    # a site far too large for one cluster stays with the streaming pipelines
+    big = layer(B, S=16, N=4096, h_in=1024, h_out=4096, dtype=1)
+    assert B.dad_compress_path(big, 16, 3)[0] in (B.DAD_PATH_GENERAL, B.DAD_PATH_TENSOR)
+    # the bounded-wait self-test checks its workspace before launching anything
+    p = ctypes.c_void_p(0x10000)
+    assert lib.dad_selftest_bounded_wait(None, 1 << 20, None) == E["DAD_ERR_NULL"]
+    assert lib.dad_selftest_bounded_wait(ctypes.c_void_p(0x10010), 1 << 20, None) == E["DAD_ERR_ALIGN"]
+    assert lib.dad_selftest_bounded_wait(p, B.DAD_SELFTEST_BYTES - 1, None) == E["DAD_ERR_WORKSPACE"]
+    # the one-term reconstruction is a valid `math`, not a valid input type
+    assert lib.dad_reconstruct(8, 8, 8, p, p, None, B.DAD_BF16_1TERM, None, 0, None) == E["DAD_ERR_NULL"]
+    assert lib.dad_reconstruct(8, 8, 8, p, p, p, 3, None, 0, None) == E["DAD_ERR_DTYPE"]
+    assert B.dad_launch_count() == before
+
+
 def test_no_cpu_fallback(B):
     """Without a CUDA device a well-formed compute call must fail with DAD_ERR_CUDA, never compute."""
     import torch
