@@ -229,6 +229,11 @@ def sweep_entries(args):
     return out
 
 
+# one more entry after those: the headline workload with ONE CALL PER LAYER instead of same-shape layers stacked per
+# call, so that the run also shows what a caller gets who does not stack
+EXTRA_ENTRY = (5, 16, 3)
+
+
 def run_ours(args):
     import copy
     import torch
@@ -256,9 +261,11 @@ def run_ours(args):
                         and not args.no_group and not args.cuda_graph and args.streams is None)
     if default_workload and not args.no_sweep and world == 1:
         sweep = []
-        for c, r, it in sweep_entries(args):
+        entries = [(e, False) for e in sweep_entries(args)] + [(EXTRA_ENTRY, True)]
+        for (c, r, it), per_layer in entries:
             a = copy.copy(args)
             a.config, a.rank, a.iters = c, r, it
+            a.no_group = per_layer
             a.no_e2e = a.no_cpu_baseline = a.no_full_grad = True
             a.steps = args.sweep_steps if c >= 4 else 20      # the launch-bound configurations take well under a millisecond
             a.warmup = max(3, args.warmup if c >= 4 else 10)
@@ -268,6 +275,7 @@ def run_ours(args):
                 keep = ("ms_per_step", "value", "unit", "steps", "warmup", "gpu_launches", "launches_per_compress", "clocks",
                         "roofline", "reconstruct", "stream_gbs", "check", "compress_path")
                 sweep.append({"config": c, "r": r, "iters": it, "workload": e["config"]["workload"],
+                              "calls": e["config"]["calls"],
                               **{k: e.get(k) for k in keep}})
         if line is not None:
             line["sweep"] = sweep

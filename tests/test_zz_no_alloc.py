@@ -40,7 +40,7 @@ def test_static_scratch_matches_reconstruct_twice_in_a_row(B, oracle):
     """Same factors through dad_reconstruct (caller workspace) and dad_reconstruct_static (library
     array), two different problems back to back: the second call finds the first one's leftovers in the
     shared array and must not be disturbed by them.  Both entry points run the same kernels on the same
-    inputs, so they must agree bit for bit; the float64 oracle's sum of outer products is the judge of
+    inputs, so they must agree bit for bit; the float64 oracle's sum of outer products decides about
     either.  From the second call on the device's free memory must not move: nothing is allocated."""
     assert torch.cuda.is_available()
     dev = torch.device("cuda:0")
