@@ -336,6 +336,21 @@ dad_status dad_check(const void* ws, void* cuda_stream);
 #define DAD_SELFTEST_BYTES (64u << 10)
 dad_status dad_selftest_bounded_wait(void* ws, size_t ws_bytes, void* cuda_stream);
 
+/*
+ * Bounds-check build (the paper has no counterpart).  Compiled with -DDAD_BOUNDS_CHECK the library is its own memory
+ * checker for the kernels that compute their indices themselves (the general products, the one-launch compress, the
+ * fp32 dense product and the small element-wise kernels; the tensor-core kernels address memory through tensor maps,
+ * which the hardware clips): dad_rank_compress, dad_full_grad, dad_gather_factors and dad_reconstruct register the
+ * address ranges of the buffers they were handed, every access of those kernels is tested against them, and an access
+ * outside all of them is NOT made (a load gives zero, a store is dropped) but counted -- nothing traps or faults.
+ *   dad_bounds_check_build  1 in such a build, 0 in the ordinary one (where the checks compile to nothing)
+ *   dad_bounds_report       synchronises `cuda_stream`, then out[0] = violations so far, out[1..3] = address, size in
+ *                           bytes and source line of the first; reset != 0 clears the record.  HOST out.  In the
+ *                           ordinary build it reports zeros.
+ */
+int dad_bounds_check_build(void);
+dad_status dad_bounds_report(uint64_t out[4], int reset, void* cuda_stream);
+
 /* Kernels launched by this library in this process so far (all threads); for accounting. */
 uint64_t dad_launch_count(void);
 

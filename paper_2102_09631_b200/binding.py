@@ -13,7 +13,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdad.so")
+# DAD_LIB picks another build of the same library (e.g. the bounds-check build libdad_check.so)
+LIB_PATH = os.path.join(_HERE, os.environ.get("DAD_LIB", "libdad.so"))
 
 DAD_OK = 0
 DAD_F32, DAD_BF16, DAD_BF16_1TERM = 0, 1, 2
@@ -28,7 +29,7 @@ EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_b
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
            "dad_rank_compress_gram", "dad_rank_compress_sequential_workspace_bytes", "dad_rank_compress_sequential",
-           "dad_check", "dad_selftest_bounded_wait", "dad_compress_path", "dad_fused_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
+           "dad_check", "dad_bounds_check_build", "dad_bounds_report", "dad_selftest_bounded_wait", "dad_compress_path", "dad_fused_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
 
@@ -110,6 +111,10 @@ def lib() -> ctypes.CDLL:
         L.dad_compress_path.restype = ctypes.c_int
         L.dad_fused_enable.argtypes = [ctypes.c_int]
         L.dad_fused_enable.restype = None
+        L.dad_bounds_check_build.argtypes = []
+        L.dad_bounds_check_build.restype = ctypes.c_int
+        L.dad_bounds_report.argtypes = [ctypes.POINTER(ctypes.c_uint64), ctypes.c_int, vp]
+        L.dad_bounds_report.restype = ctypes.c_int
         L.dad_selftest_bounded_wait.argtypes = [vp, ctypes.c_size_t, vp]
         L.dad_selftest_bounded_wait.restype = ctypes.c_int
         L.dad_check.argtypes = [vp, vp]
@@ -322,6 +327,17 @@ def dad_selftest_bounded_wait(ws, stream=None):
     """Makes one bounded device-side wait run out on purpose (nothing hangs or faults); dad_check(ws) then
     raises DAD_ERR_TIMEOUT."""
     _check(lib().dad_selftest_bounded_wait(_ptr(ws), ws.numel(), _stream(stream)), "dad_selftest_bounded_wait")
+
+
+def dad_bounds_check_build() -> bool:
+    return bool(lib().dad_bounds_check_build())
+
+
+def dad_bounds_report(reset: bool = False, stream=None):
+    """(violations, first address, bytes, source line) recorded by a -DDAD_BOUNDS_CHECK build; zeros otherwise."""
+    out = (ctypes.c_uint64 * 4)()
+    _check(lib().dad_bounds_report(out, 1 if reset else 0, _stream(stream)), "dad_bounds_report")
+    return tuple(int(x) for x in out)
 
 
 def dad_check(ws, stream=None):

@@ -26,22 +26,32 @@ def _headers():
     return glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(p) > t for p in sources() + _headers())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+CHECK_LIB = os.path.join(HERE, "libdad_check.so")
+CHECK_FLAGS = ["-DDAD_BOUNDS_CHECK", "-rdc=true"]
+
+
+def build_check(force: bool = False, verbose: bool = False) -> str:
+    """The bounds-check build of the same sources (libdad_check.so, see csrc/bounds.cuh): load it with DAD_LIB."""
+    return build(force=force, verbose=verbose, lib=CHECK_LIB, extra=CHECK_FLAGS)
+
+
+def build(force: bool = False, verbose: bool = False, lib: str = LIB, extra=None) -> str:
     """Compile every .cu under csrc/ (one object each, in parallel; an object is reused while it is newer than
     its source and every header) and link them into libdad.so; returns its path.  Raises if nvcc fails."""
-    if not force and not _stale():
+    LIB = lib
+    if not force and not _stale(LIB):
         return LIB
     from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "nvcc")
     os.makedirs(OBJ_DIR, exist_ok=True)
-    extra = os.environ.get("DAD_NVCC_EXTRA", "").split()
+    extra = list(extra or []) + os.environ.get("DAD_NVCC_EXTRA", "").split()
     tag = ("-" + "".join(c if c.isalnum() else "_" for c in " ".join(extra))) if extra else ""
     hdr_t = max(os.path.getmtime(p) for p in _headers())
     log_lines, failed = [], []
@@ -64,7 +74,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             failed.append(obj)
     tmp = LIB + f".tmp{os.getpid()}"
     if not failed:
-        cmd = [nvcc, "-shared", "-o", tmp] + objs
+        cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a"] + [x for x in extra if x.startswith("-rdc")] + ["-shared", "-o", tmp] + objs
         res = subprocess.run(cmd, capture_output=True, text=True)
         log_lines.append(" ".join(cmd) + "\n" + res.stdout + res.stderr)
         if res.returncode != 0:
@@ -81,4 +91,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--check" in sys.argv:
+        print(build_check(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

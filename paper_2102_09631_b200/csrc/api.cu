@@ -3,6 +3,7 @@
 // library; there is no host fallback.
 #include <cstring>
 
+#include "bounds.cuh"
 #include "common.cuh"
 
 namespace dad {
@@ -27,6 +28,13 @@ static dad_status validate_layer(const dad_layer* L) {
   const double big = 9.0e18;  // element counts must fit 63 bits
   if ((double)L->S * (double)L->N * (double)(L->ldA > L->ldD ? L->ldA : L->ldD) * 8.0 > big) return DAD_ERR_SHAPE;
   return DAD_OK;
+}
+
+// Bytes from the base of A (or D) to the end of its last element.
+static size_t operand_bytes(const dad_layer& L, bool isA) {
+  const size_t e = L.dtype == DAD_F32 ? 4 : 2;
+  const int64_t ld = isA ? L.ldA : L.ldD, stride = isA ? L.strideA : L.strideD, h = isA ? L.h_in : L.h_out;
+  return e * (size_t)((int64_t)(L.S - 1) * stride + (L.N - 1) * ld + h);
 }
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -321,6 +329,11 @@ dad_status dad_full_grad(const dad_layer* layer, const void* A, const void* D, f
   if (!aligned(A, 16) || !aligned(D, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
+  {
+    const BoundsRange ranges[] = {{A, operand_bytes(*L, true)}, {D, operand_bytes(*L, false)},
+                                  {grad, sizeof(float) * (size_t)L->h_in * L->h_out}, {ws, ws_bytes}};
+    if (bounds_register(ranges, 4, st) != cudaSuccess) return DAD_ERR_CUDA;
+  }
   if (tc_eligible(*L)) {
     const GemmWs w = gemm_ws_layout(L->h_in, L->h_out, L->S, L->N, false);
     if (!ws) return DAD_ERR_NULL;
@@ -356,6 +369,12 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
   if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
+  {
+    const size_t nP = sizeof(float) * (size_t)L->S * r * L->h_in, nQ = sizeof(float) * (size_t)L->S * r * L->h_out;
+    const BoundsRange ranges[] = {{A, operand_bytes(*L, true)}, {D, operand_bytes(*L, false)}, {Q0, nQ}, {P, nP}, {Q, nQ},
+                                  {sigma, sizeof(float) * (size_t)L->S * r}, {ws, ws_bytes}};
+    if (bounds_register(ranges, 7, st) != cudaSuccess) return DAD_ERR_CUDA;
+  }
   if (fused_c > 0 && g_fused_on.load(std::memory_order_relaxed)) {
     char* base = static_cast<char*>(ws);
     err = cudaMemsetAsync(base + w.status, 0, 4, st);
@@ -382,6 +401,9 @@ dad_status dad_gather_factors(const dad_layer* L, int r, const float* P, const f
   if (!aligned(P, 4) || !aligned(Q, 4) || !aligned(Pcat, 4) || !aligned(Qcat, 4)) return DAD_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (P != Pcat || Q != Qcat) {
+    const size_t nP = sizeof(float) * (size_t)L->S * r * L->h_in, nQ = sizeof(float) * (size_t)L->S * r * L->h_out;
+    const BoundsRange ranges[] = {{P, nP}, {Q, nQ}, {Pcat, nP}, {Qcat, nQ}};
+    if (bounds_register(ranges, 4, st) != cudaSuccess) return DAD_ERR_CUDA;
     cudaError_t err = copy_two(P, Pcat, (size_t)L->S * r * L->h_in, Q, Qcat, (size_t)L->S * r * L->h_out, st);
     if (err != cudaSuccess) return DAD_ERR_CUDA;
   }
@@ -420,6 +442,11 @@ dad_status dad_reconstruct_batched(int64_t h_in, int64_t h_out, int64_t K, int b
   if (!aligned(Pcat, 16) || !aligned(Qcat, 16) || !aligned(grad, 16)) return DAD_ERR_ALIGN;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaError_t err = cudaSuccess;
+  {
+    const BoundsRange ranges[] = {{Pcat, sizeof(float) * (size_t)batch * K * h_in}, {Qcat, sizeof(float) * (size_t)batch * K * h_out},
+                                  {grad, sizeof(float) * (size_t)batch * h_in * h_out}, {ws, ws_bytes}};
+    if (bounds_register(ranges, 4, st) != cudaSuccess) return DAD_ERR_CUDA;
+  }
   if (const int terms = reconstruct_terms(h_in, h_out, K, math)) {
     const GemmWs w = gemm_ws_layout(h_in, h_out, 1, terms * K, true, batch);  // `terms` bf16 products, one contraction
     if (!ws) return DAD_ERR_NULL;

@@ -15,6 +15,7 @@
 // for bit.  The only synchronisation is the hardware cluster barrier, whose release/acquire orders the remote
 // shared-memory stores; no wait is a spin.  fp32 inputs accumulate in fp64 and keep fp64 intermediates, bf16
 // inputs in fp32.
+#include "bounds.cuh"
 #include "orth_slab.cuh"
 #include "warp_reduce.cuh"
 
@@ -86,12 +87,20 @@ __host__ __device__ inline DsmGeom dsm_geom(int N, int h_in, int h_out, int r, i
 // Two adjacent input elements (a row of the site starts on an even element; widths are even), widened.
 template <typename TAcc>
 __device__ __forceinline__ void load_pair(const float* p, TAcc& a, TAcc& b) {
+  if (!DAD_RANGE_OK(p, 8)) {
+    a = b = TAcc(0);
+    return;
+  }
   const float2 t = *reinterpret_cast<const float2*>(p);
   a = TAcc(t.x);
   b = TAcc(t.y);
 }
 template <typename TAcc>
 __device__ __forceinline__ void load_pair(const __nv_bfloat16* p, TAcc& a, TAcc& b) {
+  if (!DAD_RANGE_OK(p, 4)) {
+    a = b = TAcc(0);
+    return;
+  }
   const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
   a = TAcc(t.x);
   b = TAcc(t.y);
@@ -120,11 +129,13 @@ __device__ __forceinline__ void widen_pair(__nv_bfloat162 v, TAcc& a, TAcc& b) {
 // turn a batch of requests into as many dependent round trips to L2.
 __device__ __forceinline__ float2 request_pair(const float* p) {
   float2 v;
+  if (!DAD_RANGE_OK(p, 8)) return make_float2(0.f, 0.f);
   asm volatile("ld.global.nc.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p));
   return v;
 }
 __device__ __forceinline__ __nv_bfloat162 request_pair(const __nv_bfloat16* p) {
-  uint32_t w;
+  uint32_t w = 0;
+  if (!DAD_RANGE_OK(p, 4)) return *reinterpret_cast<__nv_bfloat162*>(&w);
   asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(w) : "l"(p));
   return *reinterpret_cast<__nv_bfloat162*>(&w);
 }
@@ -238,7 +249,7 @@ __device__ __noinline__ void dsm_emit(const DsmCtx<TIn, TAcc>& cx, int sink, int
   } else if (sink == SINK_SLAB) {
     cx.slab[j * cx.Wp + cc] = v;
   } else {
-    cx.Ps[(int64_t)j * cx.h_in + c] = (float)v;
+    DAD_ST(&cx.Ps[(int64_t)j * cx.h_in + c], (float)v);
     if (sink == SINK_P_KEEP) cx.slab[j * cx.Wp + cc] = v;
   }
 }
@@ -416,12 +427,13 @@ fused_dsm_kernel(const DsmParams p) {
 #pragma unroll 1
         for (int idx = tid; idx < nrows * hv; idx += kThreads) {
           const int n = idx / hv, c = (idx - n * hv) * V;
+          if (!DAD_RANGE_OK(src + (int64_t)n * ld + c, 16)) continue;
           const uint32_t d32 = (uint32_t)__cvta_generic_to_shared(dst + (size_t)n * h + c);
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d32), "l"(src + (int64_t)n * ld + c) : "memory");
         }
       } else {
 #pragma unroll 1
-        for (int idx = tid; idx < nrows * h; idx += kThreads) dst[idx] = src[(int64_t)(idx / h) * ld + idx % h];
+        for (int idx = tid; idx < nrows * h; idx += kThreads) dst[idx] = DAD_LD(&src[(int64_t)(idx / h) * ld + idx % h]);
       }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -433,12 +445,12 @@ fused_dsm_kernel(const DsmParams p) {
 #pragma unroll 4
   for (int idx = tid; idx < rpad * hF; idx += kThreads) {
     const int j = idx / hF, c = idx - j * hF;
-    Fbuf[idx] = (j < r && c < h_out) ? TAcc(Q0s[(int64_t)j * h_out + c]) : TAcc(0);
+    Fbuf[idx] = (j < r && c < h_out) ? TAcc(DAD_LD(&Q0s[(int64_t)j * h_out + c])) : TAcc(0);
   }
   if (p.iters == 0 && p.Q != p.Q0) {
     for (int j = warp; j < r; j += kThreads / 32)
       for (int cc = lane; cc < Wg; cc += 32)
-        if (cg0 + cc < h_out) Qs[(int64_t)j * h_out + cg0 + cc] = Q0s[(int64_t)j * h_out + cg0 + cc];
+        if (cg0 + cc < h_out) DAD_ST(&Qs[(int64_t)j * h_out + cg0 + cc], DAD_LD(&Q0s[(int64_t)j * h_out + cg0 + cc]));
   }
   if (p.x_resident) asm volatile("cp.async.wait_all;" ::: "memory");
   cluster.sync();  // every CTA of the cluster is running (its shared memory may be written) and set up
@@ -464,7 +476,7 @@ fused_dsm_kernel(const DsmParams p) {
         if (c < h_out) {
           const TAcc v = slab[j * Wp + cc];
           Fbuf[j * hF + c] = v;
-          if (last) Qs[(int64_t)j * h_out + c] = (float)v;
+          if (last) DAD_ST(&Qs[(int64_t)j * h_out + c], (float)v);
         }
       }
     __syncthreads();
@@ -490,7 +502,7 @@ fused_dsm_kernel(const DsmParams p) {
         if (keep) {
           v = (double)slab[j * Wp + cc];
         } else if (cz0 + cc < h_in) {
-          v = (double)cx.Ps[(int64_t)j * h_in + cz0 + cc];  // written by this CTA above (visible after the CTA barrier)
+          v = (double)DAD_LD(&cx.Ps[(int64_t)j * h_in + cz0 + cc]);  // written by this CTA above (visible after the CTA barrier)
         }
         sq += v * v;
       }
@@ -502,7 +514,7 @@ fused_dsm_kernel(const DsmParams p) {
     if (rank == 0 && tid < r) {
       double t = 0.0;
       for (int q = 0; q < C; ++q) t += sigbuf[q * rpad + tid];
-      p.sigma[(int64_t)s * r + tid] = (float)sqrt(t);
+      DAD_ST(&p.sigma[(int64_t)s * r + tid], (float)sqrt(t));
     }
   } else {
     cluster.sync();  // no CTA leaves while a neighbour may still store into its shared memory

@@ -15,6 +15,7 @@
 //
 // Y and W live in shared memory; A_s and D_s are re-read from L2 / L1 on every pass (a site this kernel takes is a
 // few hundred KB per CTA at most).  fp32 inputs accumulate in fp64 and keep fp64 intermediates; bf16 inputs in fp32.
+#include "bounds.cuh"
 #include "orth_slab.cuh"
 #include "warp_reduce.cuh"
 
@@ -67,11 +68,11 @@ __device__ __forceinline__ void fused_rows_dot(const TIn* __restrict__ X, int64_
     for (int c = lane; c < h; c += 32) {
       TAcc x[kRowGroup];
 #pragma unroll
-      for (int q = 0; q < kRowGroup; ++q) x[q] = (row0 + q < nrows) ? TAcc(to_float(X[(int64_t)(row0 + q) * ld + c])) : TAcc(0);
+      for (int q = 0; q < kRowGroup; ++q) x[q] = (row0 + q < nrows) ? TAcc(to_float(DAD_LD(&X[(int64_t)(row0 + q) * ld + c]))) : TAcc(0);
 #pragma unroll
       for (int jj = 0; jj < kVecBlock; ++jj) {
         if (j0 + jj < r) {
-          const TAcc f = F[(int64_t)(j0 + jj) * h + c];
+          const TAcc f = DAD_LD(&F[(int64_t)(j0 + jj) * h + c]);
 #pragma unroll
           for (int q = 0; q < kRowGroup; ++q) acc[q * kVecBlock + jj] += x[q] * f;
         }
@@ -102,7 +103,7 @@ __device__ __forceinline__ void fused_cols_acc(const TIn* __restrict__ X, int64_
 #pragma unroll
         for (int g = 0; g < CG; ++g) {
           const int c = cb + g * kThreads;
-          x[g] = (c < h) ? TAcc(to_float(X[(int64_t)n * ld + c])) : TAcc(0);
+          x[g] = (c < h) ? TAcc(to_float(DAD_LD(&X[(int64_t)n * ld + c]))) : TAcc(0);
         }
 #pragma unroll
         for (int jj = 0; jj < kVecBlock; ++jj) {
@@ -117,7 +118,7 @@ __device__ __forceinline__ void fused_cols_acc(const TIn* __restrict__ X, int64_
         if (c < h) {
 #pragma unroll
           for (int jj = 0; jj < kVecBlock; ++jj)
-            if (j0 + jj < r) out[(int64_t)(j0 + jj) * h + c] = acc[g][jj];
+            if (j0 + jj < r) DAD_ST(&out[(int64_t)(j0 + jj) * h + c], acc[g][jj]);
         }
       }
     }
@@ -138,7 +139,7 @@ __device__ __forceinline__ void fused_reduce_slice(const TAcc* part_site, int64_
       if (c < h) {
         TAcc t[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) t[q] = (q < C) ? __ldcg(part_site + q * part_stride + (int64_t)j * h + c) : TAcc(0);
+        for (int q = 0; q < 8; ++q) t[q] = (q < C) ? DAD_LDCG(part_site + q * part_stride + (int64_t)j * h + c) : TAcc(0);
         v = t[0];
 #pragma unroll
         for (int q = 1; q < 8; ++q) v += t[q];
@@ -187,9 +188,9 @@ fused_site_kernel(const FusedParams p) {
     for (int cc = lane; cc < Wg; cc += 32) {
       const int c = cg0 + cc;
       if (c < h_out) {
-        const float q0 = Q0s[(int64_t)j * h_out + c];
-        FG[(int64_t)j * h_out + c] = TAcc(q0);
-        if (p.iters == 0 && p.Q != p.Q0) Qs[(int64_t)j * h_out + c] = q0;
+        const float q0 = DAD_LD(&Q0s[(int64_t)j * h_out + c]);
+        DAD_ST(&FG[(int64_t)j * h_out + c], TAcc(q0));
+        if (p.iters == 0 && p.Q != p.Q0) DAD_ST(&Qs[(int64_t)j * h_out + c], q0);
       }
     }
   cluster_barrier(cluster);
@@ -208,7 +209,7 @@ fused_site_kernel(const FusedParams p) {
     cols_acc(As, p.ldA, h_in, my_part);                                      // partial of Z = Y^T A
     cluster_barrier(cluster);
     fused_reduce_slice<TAcc>(part_site, (int64_t)r * hmax, C, r, h_in, cz0, Wz, [&](int j, int, int c, TAcc v) {
-      if (c < h_in) FZ[(int64_t)j * h_in + c] = v;
+      if (c < h_in) DAD_ST(&FZ[(int64_t)j * h_in + c], v);
     });
     cluster_barrier(cluster);
     fused_rows_dot<TIn, TAcc>(As, p.ldA, nrows, h_in, FZ, r, rpad, Ybuf);   // W = A Z^T
@@ -225,8 +226,8 @@ fused_site_kernel(const FusedParams p) {
         const int c = cg0 + cc;
         if (c < h_out) {
           const TAcc v = slab[j * Wp + cc];
-          FG[(int64_t)j * h_out + c] = v;
-          if (last) Qs[(int64_t)j * h_out + c] = (float)v;
+          DAD_ST(&FG[(int64_t)j * h_out + c], v);
+          if (last) DAD_ST(&Qs[(int64_t)j * h_out + c], (float)v);
         }
       }
     cluster_barrier(cluster);
@@ -243,7 +244,7 @@ fused_site_kernel(const FusedParams p) {
     auto flush = [&](int j) {
 #pragma unroll
       for (int o = 16; o >= 1; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-      if (lane == 0 && p.sig_part) p.sig_part[((int64_t)s * C + rank) * r + j] = sq;
+      if (lane == 0 && p.sig_part) DAD_ST(&p.sig_part[((int64_t)s * C + rank) * r + j], sq);
       sq = 0.0;
     };
     for (int j = warp; j < r; j += kThreads / 32) {
@@ -253,11 +254,11 @@ fused_site_kernel(const FusedParams p) {
         if (c < h_in) {
           TAcc t[8];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) t[q] = (q < C) ? __ldcg(part_site + (int64_t)q * r * hmax + (int64_t)j * h_in + c) : TAcc(0);
+          for (int q = 0; q < 8; ++q) t[q] = (q < C) ? DAD_LDCG(part_site + (int64_t)q * r * hmax + (int64_t)j * h_in + c) : TAcc(0);
           TAcc a = t[0];
 #pragma unroll
           for (int q = 1; q < 8; ++q) a += t[q];
-          Ps[(int64_t)j * h_in + c] = (float)a;
+          DAD_ST(&Ps[(int64_t)j * h_in + c], (float)a);
           v = (double)a;
         }
         sq += v * v;
@@ -270,8 +271,8 @@ fused_site_kernel(const FusedParams p) {
     cluster_barrier(cluster);
     if (rank == 0 && tid < r) {
       double t = 0.0;
-      for (int q = 0; q < C; ++q) t += __ldcg(p.sig_part + ((int64_t)s * C + q) * r + tid);
-      p.sigma[(int64_t)s * r + tid] = (float)sqrt(t);
+      for (int q = 0; q < C; ++q) t += DAD_LDCG(p.sig_part + ((int64_t)s * C + q) * r + tid);
+      DAD_ST(&p.sigma[(int64_t)s * r + tid], (float)sqrt(t));
     }
   }
 }

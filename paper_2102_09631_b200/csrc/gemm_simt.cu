@@ -6,6 +6,7 @@
 // Used for fp32 inputs (where bf16 tensor-core products would miss the 1e-5 parity bound) and
 // for layouts the tensor-core kernel does not take.  Also small helpers: factor gather copy,
 // fp32 -> fp64 widening, row norms.
+#include "bounds.cuh"
 #include "common.cuh"
 
 namespace dad {
@@ -35,8 +36,8 @@ gemm_tn_kernel(const TIn* __restrict__ X, int64_t ldX, int64_t strideX, const TI
       float xv = 0.f, yv = 0.f;
       if (k < Ktot) {
         const int64_t s = k / N, n = k % N;
-        if (a0 + col < hx) xv = to_float(X[s * strideX + n * ldX + a0 + col]);
-        if (b0 + col < hy) yv = to_float(Y[s * strideY + n * ldY + b0 + col]);
+        if (a0 + col < hx) xv = to_float(DAD_LD(&X[s * strideX + n * ldX + a0 + col]));
+        if (b0 + col < hy) yv = to_float(DAD_LD(&Y[s * strideY + n * ldY + b0 + col]));
       }
       Xs[kk][col] = xv;
       Ys[kk][col] = yv;
@@ -62,7 +63,7 @@ gemm_tn_kernel(const TIn* __restrict__ X, int64_t ldX, int64_t strideX, const TI
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int64_t b = b0 + tx * 4 + j;
-      if (b < hy) C[a * hy + b] = acc[i][j];
+      if (b < hy) DAD_ST(&C[a * hy + b], acc[i][j]);
     }
   }
 }
@@ -88,9 +89,9 @@ __global__ void copy_two_kernel(const float* __restrict__ a, float* __restrict__
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < na + nb; i += stride) {
     if (i < na) {
-      if (a_out != a) a_out[i] = a[i];
+      if (a_out != a) DAD_ST(&a_out[i], DAD_LD(&a[i]));
     } else {
-      if (b_out != b) b_out[i - na] = b[i - na];
+      if (b_out != b) DAD_ST(&b_out[i - na], DAD_LD(&b[i - na]));
     }
   }
 }
@@ -101,9 +102,9 @@ __global__ void copy_two_vec_kernel(const float4* __restrict__ a, float4* __rest
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < na + nb; i += stride) {
     if (i < na) {
-      if (a_out != a) a_out[i] = a[i];
+      if (a_out != a) DAD_ST(&a_out[i], DAD_LD(&a[i]));
     } else {
-      if (b_out != b) b_out[i - na] = b[i - na];
+      if (b_out != b) DAD_ST(&b_out[i - na], DAD_LD(&b[i - na]));
     }
   }
 }

@@ -6,6 +6,7 @@
 //   cols_acc : Z = Y^T X   (r x N by N x h)  -- one CTA per 128 columns, rows split over its warps and over
 //              CTAs, partial slabs summed in a fixed order by the last CTA to arrive (deterministic).
 // fp32 inputs accumulate in fp64, bf16 inputs in fp32 (TAcc).
+#include "bounds.cuh"
 #include "common.cuh"
 #include "warp_reduce.cuh"
 
@@ -48,11 +49,11 @@ rows_dot_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
     for (int64_t c = warp * 32 + lane; c < h; c += 256) {
       TAcc x[RB];
 #pragma unroll
-      for (int q = 0; q < RB; ++q) x[q] = (row0 + q < N) ? TAcc(to_float(Xs[(row0 + q) * ld + c])) : TAcc(0);
+      for (int q = 0; q < RB; ++q) x[q] = (row0 + q < N) ? TAcc(to_float(DAD_LD(&Xs[(row0 + q) * ld + c]))) : TAcc(0);
 #pragma unroll
       for (int jj = 0; jj < RT; ++jj) {
         if (j0 + jj < r) {
-          const TAcc f = Fs[(int64_t)(j0 + jj) * h + c];
+          const TAcc f = DAD_LD(&Fs[(int64_t)(j0 + jj) * h + c]);
 #pragma unroll
           for (int q = 0; q < RB; ++q) acc[q * RT + jj] += x[q] * f;
         }
@@ -67,7 +68,7 @@ rows_dot_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
 #pragma unroll
       for (int w = 1; w < 8; ++w) v += red[w][threadIdx.x];
       const int q = threadIdx.x / RT, jj = threadIdx.x % RT;
-      if (row0 + q < N && j0 + jj < r) Ys[(row0 + q) * r + j0 + jj] = v;
+      if (row0 + q < N && j0 + jj < r) DAD_ST(&Ys[(row0 + q) * r + j0 + jj], v);
     }
   }
 }
@@ -121,12 +122,12 @@ cols_acc_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int64_t c = cb + q * 32 + lane;
-        x[q] = (c < h) ? TAcc(to_float(Xs[n * ld + c])) : TAcc(0);
+        x[q] = (c < h) ? TAcc(to_float(DAD_LD(&Xs[n * ld + c]))) : TAcc(0);
       }
 #pragma unroll
       for (int jj = 0; jj < RT; ++jj) {
         if (j0 + jj < r) {
-          const TAcc y = Ys[n * r + j0 + jj];
+          const TAcc y = DAD_LD(&Ys[n * r + j0 + jj]);
 #pragma unroll
           for (int q = 0; q < 4; ++q) acc[q][jj] += y * x[q];
         }
@@ -149,8 +150,8 @@ cols_acc_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
       const int64_t c = cb + idx % kColsAccThreads;
       if (c < h && j0 + jj < r) {
         const TAcc v = red[jj][idx % kColsAccThreads];
-        dst[(int64_t)(j0 + jj) * h + c] = v;
-        if (splits == 1 && out32) out32[((int64_t)s * r + j0 + jj) * h + c] = (float)v;
+        DAD_ST(&dst[(int64_t)(j0 + jj) * h + c], v);
+        if (splits == 1 && out32) DAD_ST(&out32[((int64_t)s * r + j0 + jj) * h + c], (float)v);
       }
     }
     __syncthreads();
@@ -179,13 +180,13 @@ cols_acc_kernel(const TIn* __restrict__ X, int64_t ld, int64_t stride, int64_t N
     for (; p + 4 <= splits; p += 4) {  // four loads in flight, added in split order
       TAcc t[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) t[u] = __ldcg(src + ((int64_t)(p + u) * r + j) * h + c);
+      for (int u = 0; u < 4; ++u) t[u] = DAD_LDCG(src + ((int64_t)(p + u) * r + j) * h + c);
 #pragma unroll
       for (int u = 0; u < 4; ++u) v += t[u];
     }
-    for (; p < splits; ++p) v += __ldcg(src + ((int64_t)p * r + j) * h + c);
-    Zs[(int64_t)j * h + c] = v;
-    if (out32) out32[((int64_t)s * r + j) * h + c] = (float)v;
+    for (; p < splits; ++p) v += DAD_LDCG(src + ((int64_t)p * r + j) * h + c);
+    DAD_ST(&Zs[(int64_t)j * h + c], v);
+    if (out32) DAD_ST(&out32[((int64_t)s * r + j) * h + c], (float)v);
   }
 }
 

@@ -167,6 +167,31 @@ def test_one_launch_compress_matches_oracle_and_the_multi_launch_pipeline(oracle
     assert rel(g1["grad"], g3["grad"]) <= tol
 
 
+@pytest.mark.parametrize("S,N,h_in,h_out,r,iters,dtype", [(3, 40, 64, 48, 4, 2, torch.float32),      # one-launch, on chip
+                                                          (3, 70, 264, 520, 40, 2, torch.float32),   # one-launch, through L2
+                                                          (2, 300, 256, 512, 16, 2, torch.bfloat16),  # tensor-core pipeline
+                                                          (3, 2000, 96, 40, 5, 1, torch.float32)])   # general pipeline
+def test_q_may_alias_the_start_block(oracle, B, S, N, h_in, h_out, r, iters, dtype):
+    """dad_rank_compress allows Q == Q0 (the start vectors are overwritten by the result): every pipeline gives,
+    bit for bit, what it gives with separate buffers."""
+    dev = torch.device("cuda:0")
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 61 + N, dtype, dev)
+    Q0 = wl.start_block(S, r, h_out, 61 + N, dev)
+    L = B.make_layer(A, D)
+    ws = B.new_workspace(B.dad_workspace_bytes(L, r, iters), dev)
+    P1, Q1 = torch.empty(S, r, h_in, device=dev), torch.empty(S, r, h_out, device=dev)
+    sg1 = torch.empty(S, r, device=dev)
+    B.dad_rank_compress(L, A, D, r, iters, Q0, P1, Q1, sg1, ws)
+    B.dad_check(ws)
+    P2, Q2, sg2 = torch.empty_like(P1), Q0.clone(), torch.empty_like(sg1)
+    B.dad_rank_compress(L, A, D, r, iters, Q2, P2, Q2, sg2, ws)
+    B.dad_check(ws)
+    assert torch.equal(P1, P2) and torch.equal(Q1, Q2) and torch.equal(sg1, sg2)
+    Po, Qo, _ = oracle.spi_block(A[:1].cpu(), D[:1].cpu(), Q0[:1].cpu(), iters)
+    got = P2[0].double().cpu().numpy().T @ Q2[0].double().cpu().numpy()
+    assert rel(got, Po[0].T @ Qo[0]) <= TOL[dtype]
+
+
 def test_config1_single_linear_layer(oracle, B):
     cfg = wl.CONFIGS[1]
     A, D, Q0 = wl.layer_inputs(cfg, cfg.layers[0], 0)
