@@ -674,7 +674,7 @@ def measure(args, rank, local, world, dev, headline):
     torch.cuda.synchronize()
     launches_per_compress = B.dad_launch_count() - c0
     names = {B.DAD_PATH_GENERAL: "general", B.DAD_PATH_TENSOR: "tensor", B.DAD_PATH_FUSED: "fused",
-             B.DAD_PATH_FUSED_L2: "fused_l2"}
+             B.DAD_PATH_FUSED_L2: "fused_l2", B.DAD_PATH_TENSOR_PAIRED: "tensor_paired"}
     compress_path = {f"{k[0]}->{k[1]} x{k[2]}": names.get(B.dad_compress_path(pl.layer, r, iters)[0], "?")
                      for k, pl in plans.items()}
     check = None

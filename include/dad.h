@@ -140,9 +140,13 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
 
 /*
  * Which of the library's pipelines dad_rank_compress takes for this shape (informational; the paper has no
- * counterpart).  All three compute the iteration stated above to the same precision contract:
+ * counterpart).  All of them compute the iteration stated above to the same precision contract:
  *   DAD_PATH_GENERAL  any shape: one launch per product and per Cholesky-QR phase (5 * iters + 3 or more launches)
  *   DAD_PATH_TENSOR   bf16 inputs in 16-byte-aligned layouts: the same sequence on tcgen05 tensor cores
+ *   DAD_PATH_TENSOR_PAIRED  the tensor-core sequence for calls of few row blocks with each half of the operator of
+ *                     Eq. "reduced_iter" (Y = D g then Z = Y^T A; W = A Z^T then W^T D) as one launch in which Y / W
+ *                     never leaves the SM (2 * iters + 1 product launches instead of 4 * iters + 2); an option,
+ *                     taken only after dad_pair_enable(1)
  *   DAD_PATH_FUSED    small sites: ONE launch, a thread-block cluster of *cluster_size CTAs per site runs every
  *                     application of the operator, the orthonormalisations and the final factor, with Y and W
  *                     in shared memory and Z, G~ and the orthonormal vectors exchanged over distributed shared
@@ -151,14 +155,18 @@ dad_status dad_rank_compress(const dad_layer* layer, const void* A, const void* 
  *                     sums and factors through the workspace (L2) instead.
  * Returns -1 for invalid arguments; cluster_size may be NULL.  dad_fused_enable(0) makes the library skip the
  * one-launch form (process-wide; for timing one pipeline against the other), dad_fused_enable(1) restores it.
- * The workspace size does not depend on that switch.
+ * The workspace size does not depend on that switch.  dad_pair_enable(1 / 0) switches the paired launches of the
+ * tensor-core sequence on and off (process-wide; off by default: on B200 they measured no faster than the two
+ * streaming kernels they replace); the workspace size does not depend on it either.
  */
 #define DAD_PATH_GENERAL 0
 #define DAD_PATH_TENSOR 1
 #define DAD_PATH_FUSED 2
 #define DAD_PATH_FUSED_L2 3
+#define DAD_PATH_TENSOR_PAIRED 4
 int dad_compress_path(const dad_layer* layer, int r, int iters, int* cluster_size);
 void dad_fused_enable(int on);
+void dad_pair_enable(int on);
 
 /*
  * The same compression in the form Algorithm 2 prints it, for the regime the paper assumes (batch much smaller

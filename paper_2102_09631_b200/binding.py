@@ -29,7 +29,7 @@ EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_b
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
            "dad_rank_dad_host_scratch_bytes", "dad_rank_dad_host", "dad_rank_compress_gram_workspace_bytes",
            "dad_rank_compress_gram", "dad_rank_compress_sequential_workspace_bytes", "dad_rank_compress_sequential",
-           "dad_check", "dad_bounds_check_build", "dad_bounds_report", "dad_selftest_bounded_wait", "dad_compress_path", "dad_fused_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
+           "dad_check", "dad_bounds_check_build", "dad_bounds_report", "dad_selftest_bounded_wait", "dad_compress_path", "dad_fused_enable", "dad_pair_enable", "dad_launch_count", "dad_status_string", "dad_timing_enable", "dad_timing_collect",
            "dad_timing_reset", "dad_timing_name", "dad_timing_ms", "dad_timing_launches"]
 
 
@@ -111,6 +111,8 @@ def lib() -> ctypes.CDLL:
         L.dad_compress_path.restype = ctypes.c_int
         L.dad_fused_enable.argtypes = [ctypes.c_int]
         L.dad_fused_enable.restype = None
+        L.dad_pair_enable.argtypes = [ctypes.c_int]
+        L.dad_pair_enable.restype = None
         L.dad_bounds_check_build.argtypes = []
         L.dad_bounds_check_build.restype = ctypes.c_int
         L.dad_bounds_report.argtypes = [ctypes.POINTER(ctypes.c_uint64), ctypes.c_int, vp]
@@ -186,7 +188,7 @@ def dad_workspace_bytes(layer: dad_layer, r: int, iters: int) -> int:
     return int(lib().dad_workspace_bytes(ctypes.byref(layer), r, iters))
 
 
-DAD_PATH_GENERAL, DAD_PATH_TENSOR, DAD_PATH_FUSED, DAD_PATH_FUSED_L2 = 0, 1, 2, 3
+DAD_PATH_GENERAL, DAD_PATH_TENSOR, DAD_PATH_FUSED, DAD_PATH_FUSED_L2, DAD_PATH_TENSOR_PAIRED = 0, 1, 2, 3, 4
 
 
 def dad_compress_path(layer: dad_layer, r: int, iters: int):
@@ -197,6 +199,11 @@ def dad_compress_path(layer: dad_layer, r: int, iters: int):
 
 def dad_fused_enable(on: bool):
     lib().dad_fused_enable(1 if on else 0)
+
+
+def dad_pair_enable(on: bool):
+    """Process-wide switch of the paired launches of the tensor-core sequence (for timing one form against the other)."""
+    lib().dad_pair_enable(1 if on else 0)
 
 
 def dad_launch_count() -> int:

@@ -10,6 +10,7 @@ namespace dad {
 
 std::atomic<uint64_t> g_launches{0};
 static std::atomic<bool> g_fused_on{true};
+static std::atomic<bool> g_pair_on{false};
 
 static bool layer_ok(const dad_layer* L) {
   if (!L) return false;
@@ -66,7 +67,10 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc, int 
   size_t off = 0;
   w.status = off;
   off += 256;
-  w.n_counters = S * (size_t)ceil_div((int64_t)hmax, kColsAccThreads) + S;
+  // arrival counters: column tiles of the split products | chunks of the one-launch pairs | sites (Gram kernel)
+  const bool pair_in = tc && umma_pair_fits(L.S, L.N, L.h_in, r), pair_out = tc && umma_pair_fits(L.S, L.N, L.h_out, r);
+  w.n_pair_counters = (pair_in || pair_out) ? S * 16 : 0;
+  w.n_counters = S * (size_t)ceil_div((int64_t)hmax, kColsAccThreads) + w.n_pair_counters + S;
   w.counters = off;
   off = align_up(off + w.n_counters * sizeof(unsigned), 256);
   w.G = off;
@@ -104,7 +108,10 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc, int 
     const size_t p_in = (size_t)umma_cols_acc_splits(L.S, L.N, L.h_in) * (size_t)ceil_div(L.h_in, 128);
     const size_t p_out = (size_t)umma_cols_acc_splits(L.S, L.N, L.h_out) * (size_t)ceil_div(L.h_out, 128);
     w.tc_partial = off;
-    off = align_up(off + S * (p_in > p_out ? p_in : p_out) * 128 * rp * 4, 256);
+    size_t part_bytes = S * (p_in > p_out ? p_in : p_out) * 128 * rp * 4;
+    if (pair_in && umma_pair_partial_bytes(L.S, L.N, L.h_in, r) > part_bytes) part_bytes = umma_pair_partial_bytes(L.S, L.N, L.h_in, r);
+    if (pair_out && umma_pair_partial_bytes(L.S, L.N, L.h_out, r) > part_bytes) part_bytes = umma_pair_partial_bytes(L.S, L.N, L.h_out, r);
+    off = align_up(off + part_bytes, 256);
   }
   w.fused_part = w.fused_sig = off;
   if (fused_c > 0) {
@@ -215,6 +222,7 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
   int* status = reinterpret_cast<int*>(ws + w.status);
   unsigned* ctr_cols = reinterpret_cast<unsigned*>(ws + w.counters);
   unsigned* ctr_gram = ctr_cols + (w.n_counters - (size_t)S);
+  unsigned* ctr_pair = ctr_gram - w.n_pair_counters;
   double* gram_partial = reinterpret_cast<double*>(ws + w.gram_partial);
   double* gram = reinterpret_cast<double*>(ws + w.gram);
   double* tratio = reinterpret_cast<double*>(ws + w.tratio);
@@ -238,13 +246,28 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
             make_tmap_bf16_3d(&tmYt, Yt, N, rp, (uint64_t)S * 2, (uint64_t)w.Npad * 2, (uint64_t)rp * w.Npad * 2, 64, rp);
   if (!ok) return cudaErrorInvalidValue;
 
+  // Small calls take each half of the operator (Y = D G^T, Z = Y^T A; W = A Z^T, G~ = W^T D) as ONE launch in which Y
+  // (or W) stays on the SM; large ones as the two streaming kernels with Y^T handed on through the workspace.
+  const bool pair_on = g_pair_on.load(std::memory_order_relaxed);
+  const bool pair_in = pair_on && umma_pair_fits(S, N, hi, r), pair_out = pair_on && umma_pair_fits(S, N, ho, r);
+  auto half_in = [&](float* out32, __nv_bfloat16* planes) -> cudaError_t {  // (D G^T)^T A from the planes Fq
+    if (pair_in) return umma_pair(tmD_rows, tmFq, tmA_cols, S, N, ho, hi, r, out32, nullptr, planes, hi, part, ctr_pair, status, st);
+    cudaError_t e = umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st);
+    if (e != cudaSuccess) return e;
+    return umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, out32, nullptr, planes, hi, part, ctr_cols, status, st);
+  };
+  auto half_out = [&]() -> cudaError_t {  // (A Z^T)^T D from the planes Fz, into Q
+    if (pair_out) return umma_pair(tmA_rows, tmFz, tmD_cols, S, N, hi, ho, r, Q, nullptr, nullptr, 0, part, ctr_pair, status, st);
+    cudaError_t e = umma_rows_dot(tmA_rows, tmFz, S, N, hi, r, Yt, w.Npad, status, st);
+    if (e != cudaSuccess) return e;
+    return umma_cols_acc(tmD_cols, tmYt, S, N, ho, r, Q, nullptr, nullptr, 0, part, ctr_cols, status, st);
+  };
+
   if (Q != Q0) DAD_STEP(cudaMemcpyAsync(Q, Q0, sizeof(float) * (size_t)S * r * ho, cudaMemcpyDeviceToDevice, st));
   DAD_STEP(split_planes(Q0, S, r, ho, Fq, rp, st));
   for (int k = 0; k < iters; ++k) {
-    DAD_STEP(umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st));                                  // Y = D G^T
-    DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, nullptr, nullptr, Fz, hi, part, ctr_cols, status, st));     // Z = Y^T A
-    DAD_STEP(umma_rows_dot(tmA_rows, tmFz, S, N, hi, r, Yt, w.Npad, status, st));                                  // W = A Z^T
-    DAD_STEP(umma_cols_acc(tmD_cols, tmYt, S, N, ho, r, Q, nullptr, nullptr, 0, part, ctr_cols, status, st));       // Gt = W^T D
+    DAD_STEP(half_in(nullptr, Fz));
+    DAD_STEP(half_out());
     if (orth_split_preferred(r, ho, S)) {
       DAD_STEP(orth_split(Q, S, r, ho, tol, gram_partial, gram, tratio, dead, need2, ctr_gram, status, nullptr, Fq, rp, st));
     } else if (orth_mma_fits(r, ho)) {
@@ -258,8 +281,7 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
                                   nullptr, Fq, rp, st));
     }
   }
-  DAD_STEP(umma_rows_dot(tmD_rows, tmFq, S, N, ho, r, Yt, w.Npad, status, st));
-  DAD_STEP(umma_cols_acc(tmA_cols, tmYt, S, N, hi, r, P, nullptr, nullptr, 0, part, ctr_cols, status, st));
+  DAD_STEP(half_in(P, nullptr));
   if (sigma) DAD_STEP(row_norms<float>(P, (int64_t)S * r, hi, sigma, st));
   return cudaSuccess;
 }
@@ -491,10 +513,14 @@ int dad_compress_path(const dad_layer* layer, int r, int iters, int* cluster_siz
     if (cluster_size) *cluster_size = c;
     return fused_dsm_fits(L, r, c, nullptr) ? DAD_PATH_FUSED : DAD_PATH_FUSED_L2;
   }
-  return tc_eligible(L) ? DAD_PATH_TENSOR : DAD_PATH_GENERAL;
+  if (!tc_eligible(L)) return DAD_PATH_GENERAL;
+  const bool paired = g_pair_on.load(std::memory_order_relaxed) &&
+                      (umma_pair_fits(L.S, L.N, L.h_in, r) || umma_pair_fits(L.S, L.N, L.h_out, r));
+  return paired ? DAD_PATH_TENSOR_PAIRED : DAD_PATH_TENSOR;
 }
 
 void dad_fused_enable(int on) { g_fused_on.store(on != 0, std::memory_order_relaxed); }
+void dad_pair_enable(int on) { g_pair_on.store(on != 0, std::memory_order_relaxed); }
 
 dad_status dad_selftest_bounded_wait(void* ws, size_t ws_bytes, void* cuda_stream) {
   if (!ws) return DAD_ERR_NULL;

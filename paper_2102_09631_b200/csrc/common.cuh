@@ -69,6 +69,7 @@ struct CompressWs {
   size_t status;        // int32 status word (+ padding)
   size_t counters;      // uint32 arrival counters of the split reductions
   size_t n_counters;
+  size_t n_pair_counters;  // of those: chunk counters of the one-launch pairs (before the last S, the Gram kernel's)
   size_t G;             // S*r*h_out accumulator-type iterate (fp64 pipeline only)
   size_t Y;             // S*N*r
   size_t Z;             // S*r*h_in
@@ -189,6 +190,12 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
 cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,
                           float* out2, __nv_bfloat16* planes, int64_t ld_planes, float* partial, unsigned* counters,
                           int* status, cudaStream_t st);
+// One launch for the pair Z = (X1 F^T)^T X2 (umma_pair.cu): whether it takes a shape, the partial blocks it needs, launch.
+bool umma_pair_fits(int S, int64_t N, int64_t h2, int r);
+size_t umma_pair_partial_bytes(int S, int64_t N, int64_t h2, int r);
+cudaError_t umma_pair(const CUtensorMap& tmX1, const CUtensorMap& tmF, const CUtensorMap& tmX2, int S, int64_t N, int64_t h1,
+                      int64_t h2, int r, float* out, float* out2, __nv_bfloat16* planes, int64_t ld_planes, float* partial,
+                      unsigned* counters, int* status, cudaStream_t st);
 cudaError_t umma_selftest_timeout(char* area, int* status, cudaStream_t st);
 cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& plan, int64_t hx, int64_t hy,
                          float* C, float* partial, unsigned* counters, int* status, cudaStream_t st);

@@ -1002,10 +1002,20 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
   p.plane_rows = umma_rank_pad(r);
   p.status = status;
   dim3 grid((unsigned)ceil_div(N, 128), 1, (unsigned)S);
+  // A launch of at most one or two CTAs per SM has no neighbours to cover a CTA's load latency: there the CTA keeps
+  // eight (or four) stages in flight itself (64 CTAs streaming 2048-wide rows: 17.4 us with two stages).
+  const int64_t ctas = (int64_t)grid.x * grid.z;
   switch (umma_rank_pad(r)) {
-    case 16: return launch_umma<16, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
-    case 32: return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
-    default: return launch_umma<64, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    case 16:
+      if (ctas <= 148) return launch_umma<16, false, false, 2, EPI_YT, 8>(tmX, tmF, p, grid, "rows_dot_tc", st);
+      if (ctas <= 2 * 148) return launch_umma<16, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
+      return launch_umma<16, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    case 32:
+      if (ctas <= 148) return launch_umma<32, false, false, 2, EPI_YT, 8>(tmX, tmF, p, grid, "rows_dot_tc", st);
+      return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    default:
+      if (ctas <= 148) return launch_umma<64, false, false, 2, EPI_YT, 6>(tmX, tmF, p, grid, "rows_dot_tc", st);
+      return launch_umma<64, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
   }
 }
 

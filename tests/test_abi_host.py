@@ -148,7 +148,7 @@ def test_pipeline_query_and_diagnostics_validate_their_arguments(B):
         B.dad_fused_enable(True)
     # a site far too large for one cluster stays with the streaming pipelines
     big = layer(B, S=16, N=4096, h_in=1024, h_out=4096, dtype=1)
-    assert B.dad_compress_path(big, 16, 3)[0] in (B.DAD_PATH_GENERAL, B.DAD_PATH_TENSOR)
+    assert B.dad_compress_path(big, 16, 3)[0] in (B.DAD_PATH_GENERAL, B.DAD_PATH_TENSOR, B.DAD_PATH_TENSOR_PAIRED)
     # the bounded-wait self-test checks its workspace before launching anything
     p = ctypes.c_void_p(0x10000)
     assert lib.dad_selftest_bounded_wait(None, 1 << 20, None) == E["DAD_ERR_NULL"]

@@ -158,7 +158,7 @@ def test_one_launch_compress_matches_oracle_and_the_multi_launch_pipeline(oracle
     assert np.array_equal(g1["P"], g2["P"]) and np.array_equal(g1["Q"], g2["Q"]) and np.array_equal(g1["sigma"], g2["sigma"])
     B.dad_fused_enable(False)
     try:
-        assert B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)[0] in (B.DAD_PATH_GENERAL, B.DAD_PATH_TENSOR)
+        assert B.dad_compress_path(B.make_layer(A.to(dev), D.to(dev)), r, iters)[0] in (B.DAD_PATH_GENERAL, B.DAD_PATH_TENSOR, B.DAD_PATH_TENSOR_PAIRED)
         g3 = run_gpu_layer(B, A, D, Q0, r, iters)
     finally:
         B.dad_fused_enable(True)
@@ -224,6 +224,44 @@ def test_config3_encoder_layer_projections(oracle, B):
         assert A.dtype == torch.bfloat16 and A.shape[1] == cfg.N
         Q0 = wl.start_block(cfg.S, cfg.r, D.shape[2], wl.seed_for(3, i))
         check_layer(oracle, B, A, D, Q0, cfg.r, cfg.iters, TOL[torch.bfloat16], ortho_tol=1e-3)
+
+
+@pytest.mark.parametrize("S,N,h_in,h_out,r,iters", [
+    (4, 2048, 512, 2048, 10, 3),    # configuration 3's widest layer: 16 chunks fill tensor memory in one direction
+    (16, 2048, 512, 512, 10, 2),    # its attention projections stacked as 16 slices: two shallow CTAs per SM
+    (3, 1000, 200, 136, 7, 2),      # rows no multiple of 64 or 128, widths of no tile, rank below the padded 16
+    (2, 100, 264, 520, 24, 2),      # one row block per site (nothing to sum), rank padded to 32
+    (5, 333, 1024, 776, 32, 1),     # rank 32 at the widest X2 it takes (8 chunks of 64 columns of tensor memory)
+    (2, 700, 768, 3072, 16, 2),     # paired in one direction only: the 3072-wide half keeps the two streaming kernels
+])
+def test_paired_launches_match_the_oracle_and_the_two_kernel_sequence(oracle, B, S, N, h_in, h_out, r, iters):
+    """Calls of few row blocks can run each half of the operator of Eq. "reduced_iter" as one launch (Y stays on the SM;
+    dad_pair_enable): parity with the oracle, two runs bit for bit (the partial blocks are summed in row-block order), and agreement with
+    the two-kernel sequence on the same inputs far inside the bar."""
+    dev = torch.device("cuda:0")
+    seed = 3100 + N + h_out
+    A, D = wl.decaying_layer(S, N, h_in, h_out, seed, torch.bfloat16)
+    Q0 = wl.start_block(S, r, h_out, seed)
+    L = B.make_layer(A.to(dev), D.to(dev))
+    tol = TOL[torch.bfloat16]
+    B.dad_fused_enable(False)    # the smallest of these sites would otherwise take the one-launch cluster form
+    B.dad_pair_enable(True)      # the paired launches are an option (off by default: measured no faster, see the kernel's header)
+    try:
+        assert B.dad_compress_path(L, r, iters)[0] == B.DAD_PATH_TENSOR_PAIRED
+        g1, o = check_layer(oracle, B, A, D, Q0, r, iters, tol, ortho_tol=1e-3)
+        for s in range(S):
+            assert rel(g1["P"][s].T @ g1["Q"][s], o["P"][s].T @ o["Q"][s]) <= 1e-4   # what the path delivers, not only the bar
+        g2 = run_gpu_layer(B, A, D, Q0, r, iters)
+        assert np.array_equal(g1["P"], g2["P"]) and np.array_equal(g1["Q"], g2["Q"]) and np.array_equal(g1["sigma"], g2["sigma"])
+        B.dad_pair_enable(False)
+        assert B.dad_compress_path(L, r, iters)[0] == B.DAD_PATH_TENSOR
+        g3 = run_gpu_layer(B, A, D, Q0, r, iters)
+    finally:
+        B.dad_pair_enable(False)
+        B.dad_fused_enable(True)
+    for s in range(S):
+        assert rel(g1["P"][s].T @ g1["Q"][s], g3["P"][s].T @ g3["Q"][s]) <= 1e-4
+    assert rel(g1["grad"], g3["grad"]) <= 1e-4
 
 
 @pytest.mark.parametrize("N,h_in,h_out,r,iters,dtype", [
