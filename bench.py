@@ -576,6 +576,9 @@ def measure(args, rank, local, world, dev, headline):
                        "ms_per_step": rec["ms_per_step"], "tflops_algorithmic": flops / t / 1e12,
                        "tflops_executed": tf_exec,
                        "frac_tensor_executed": tf_exec / peaks["bf16_tflops"] if bf16 else None,
+                       # the product is timed inside the step's event pass, i.e. under the power cap of a long run: its
+                       # measured counterpart is the sustained cuBLAS figure, given beside the burst one above
+                       "frac_tensor_executed_of_sustained": tf_exec / peaks["bf16_tflops_sustained"] if bf16 else None,
                        "gbs": (out_bytes + in_bytes) / t / 1e9, "frac_hbm": (out_bytes + in_bytes) / t / 1e9 / peaks["hbm_gbs"],
                        "bound": "tensor" if bf16 and terms * flops / (peaks["bf16_tflops"] * 1e12) >
                                 (out_bytes + in_bytes) / (peaks["hbm_gbs"] * 1e9) else "hbm"}

@@ -20,6 +20,8 @@
 // Every mbarrier wait is bounded; if one runs out the CTA raises an abort flag, all roles leave
 // their loops, outstanding copies are waited for (bounded), tensor memory is freed, and the status
 // word in the workspace is set to DAD_ERR_TIMEOUT.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "umma.cuh"
 
@@ -829,6 +831,221 @@ umma_gemm_persist_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 }
 
 
+// Dense product C = X^T Y for short contractions, persistent form on CTA PAIRS (cta_group::2): two CTAs of a cluster,
+// on neighbouring SMs, own a 256 x 256 output tile together.  Each loads its own 128 columns of X (rows of the tile)
+// and only HALF of the tile's 256 columns of Y per 64-deep block -- 32 KB instead of the 48 KB a lone CTA needs for a
+// 128 x 256 tile -- and the tensor cores of both SMs read the two halves of Y out of both shared memories.  The
+// reconstruction (Algorithm 1, P^T Q) is bound by exactly those bytes: at a contraction of a few hundred rows a CTA
+// spends longer pulling its operands through its SM's L2 port than multiplying or storing.  One thread of the leader
+// (cluster rank 0) issues the MMAs for both CTAs; every CTA fetches its own tiles with plain TMA loads (no cluster
+// multicast), whose completion is counted on the leader's barrier; a commit arrives on the barriers of both CTAs.
+// Each CTA holds two accumulators of 128 x 256 in its tensor memory, so the epilogue of one tile (through two staging
+// boxes and TMA stores, as in umma_gemm_persist_kernel) runs under the MMAs of the next.  Waits are bounded as
+// everywhere; whatever happens, every thread of both CTAs reaches the cluster barrier before tensor memory is freed.
+template <int STAGES>
+__global__ void __launch_bounds__(192)
+umma_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
+  constexpr int A_BYTES = 2 * 8192, B_BYTES = 2 * 8192, STAGE_BYTES = A_BYTES + B_BYTES;  // per CTA
+  constexpr int BOX_BYTES = 128 * 128;  // [128 rows][32 fp32]
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t IDESC = instr_desc(256, 256, true, true);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* boxes = smem + (size_t)STAGES * STAGE_BYTES;
+  // full / acc_empty are used in the leader only (they count both CTAs); empty / acc_full in each CTA
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2], flush_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag, issued_s, flush_s, epi_bad;
+  const uint32_t wlim = p.wait_limit ? p.wait_limit : kWaitLimit;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int per_product = p.tiles_m * p.tiles_n;  // 256 x 256 tiles
+  const int n_tiles = per_product * p.batch_count;
+  const int nkb = p.k_blocks;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 256);  // the epilogue threads of both CTAs
+    }
+    mbar_init(&flush_bar, 1);
+    abort_flag = 0;
+    issued_s = 0;
+    flush_s = 0;
+    epi_bad = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(&tmem_base_s, TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_barrier_all();  // both CTAs' barriers are initialised before either signals the other's
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  volatile int* abortp = &abort_flag;
+
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // tile t: product t / per_product; inside it m fastest, so that pairs working side by side share a panel of Y
+  auto tile_at = [&](int t, int& m0, int& n0, int& bz) {
+    bz = t / per_product;
+    const int rem = t - bz * per_product;
+    n0 = (rem / p.tiles_m) * 256;
+    m0 = (rem % p.tiles_m) * 256;
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmA);
+      prefetch_tmap(&tmB);
+      int g = 0;
+      bool go = true;
+      for (int t = pair; go && t < n_tiles; t += n_pairs) {
+        int m0, n0, bz;
+        tile_at(t, m0, n0, bz);
+        m0 += 128 * (int)rank;  // this CTA's rows of the tile
+        n0 += 128 * (int)rank;  // ... and its half of the tile's columns of Y
+        for (int kb = 0; kb < nkb; ++kb, ++g) {
+          const int stage = g % STAGES;
+          const uint32_t ph = (uint32_t)(g / STAGES) & 1u;
+          if (!mbar_wait(&empty_bar[stage], ph ^ 1u, abortp, wlim)) {
+            go = false;
+            break;
+          }
+          if (leader) mbar_expect_tx(&full_bar[stage], 2 * STAGE_BYTES);  // the tiles of both CTAs
+          const uint32_t bar = cluster_map(smem_u32(&full_bar[stage]), 0);
+          uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_BYTES;
+          const int kcoord = kb * 64;
+          tma_load_3d_pair(a_dst, &tmA, bar, m0, kcoord, bz);
+          tma_load_3d_pair(a_dst + 8192, &tmA, bar, m0 + 64, kcoord, bz);
+          tma_load_3d_pair(b_dst, &tmB, bar, n0, kcoord, bz);
+          tma_load_3d_pair(b_dst + 8192, &tmB, bar, n0 + 64, kcoord, bz);
+          issued_s = g + 1;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      int g = 0, it = 0;
+      bool go = true;
+      for (int t = pair; go && t < n_tiles; t += n_pairs, ++it) {
+        const int buf = it & 1;
+        const uint32_t uses = (uint32_t)(it >> 1);
+        // both epilogues have read this accumulator's previous tile out (passes at once on its first use)
+        if (!mbar_wait(&acc_empty[buf], (uses & 1u) ^ 1u, abortp, wlim)) break;
+        tc_fence_after();
+        const uint32_t acc = tmem_base + (uint32_t)buf * 256u;
+        for (int kb = 0; kb < nkb; ++kb, ++g) {
+          const int stage = g % STAGES;
+          const uint32_t ph = (uint32_t)(g / STAGES) & 1u;
+          if (!mbar_wait(&full_bar[stage], ph, abortp, wlim)) {
+            go = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k16 = 0; k16 < 4; ++k16)
+            umma_bf16_pair(acc, desc_mn_major(a_addr, k16), desc_mn_major(b_addr, k16), IDESC, (kb | k16) != 0 ? 1u : 0u);
+          umma_commit_pair(&empty_bar[stage]);
+        }
+        if (go) umma_commit_pair(&acc_full[buf]);
+      }
+      if (*abortp) {  // giving up: the teardown waits on this for the MMAs issued so far before tensor memory is freed
+        umma_commit_pair(&flush_bar);
+        flush_s = 1;
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const bool issuer = warp == 2 && lane == 0;
+    if (issuer) prefetch_tmap(&tmC);
+    int it = 0, boxes_used = 0;
+    for (int t = pair; t < n_tiles; t += n_pairs, ++it) {
+      int m0, n0, bz;
+      tile_at(t, m0, n0, bz);
+      m0 += 128 * (int)rank;
+      const int buf = it & 1;
+      const uint32_t uses = (uint32_t)(it >> 1);
+      if (!mbar_wait(&acc_full[buf], uses & 1u, abortp, wlim)) epi_bad = 1;
+      asm volatile("bar.sync 1, 128;" ::: "memory");  // the four warps go on, or stop, together
+      if (*reinterpret_cast<volatile int*>(&epi_bad)) break;
+      tc_fence_after();
+      const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
+#pragma unroll 1
+      for (int c32 = 0; c32 < 8; ++c32, ++boxes_used) {
+        uint8_t* box = boxes + (boxes_used & 1) * BOX_BYTES;
+        if (boxes_used >= 2) {  // the store that read this box two rounds ago has to be done with it
+          if (issuer) bulk_wait_read<1>();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        float v[32];
+        tmem_ld16(lane_base + c32 * 32, *reinterpret_cast<float(*)[16]>(&v[0]));
+        tmem_ld16(lane_base + c32 * 32 + 16, *reinterpret_cast<float(*)[16]>(&v[16]));
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          *reinterpret_cast<float4*>(box + row * 128 + ((k ^ (row & 7)) * 16)) =
+              make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+        fence_async_proxy();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (issuer) {
+          if (n0 + c32 * 32 < p.n_extent && m0 < p.m_extent) tma_store_3d(&tmC, box, n0 + c32 * 32, m0, bz);
+          bulk_commit();  // (an empty group where the box lies beyond C, so that the count of groups stays in step)
+        }
+      }
+      // this thread's part of the accumulator is in shared memory: the tensor cores may overwrite it
+      tc_fence_before();
+      mbar_arrive_remote(cluster_map(smem_u32(&acc_empty[buf]), 0));
+    }
+    if (issuer) bulk_wait_all();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  // Neither CTA goes on to free tensor memory, or leaves, while its peer may still read its shared memory, arrive on
+  // its barriers or multiply into its accumulators.
+  if (abort_flag) {
+    if (threadIdx.x == 0) {
+      const int issued = issued_s;
+      const int first = issued > STAGES ? issued - STAGES : 0;
+      if (leader) {
+        for (int i = first; i < issued; ++i) {
+          uint64_t* bar = &full_bar[i % STAGES];
+          const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+          for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(bar, ph); ++t) {
+          }
+        }
+      }
+      if (flush_s) {
+        for (uint32_t t = 0; t < kWaitLimit && !mbar_try_wait(&flush_bar, 0u); ++t) {
+        }
+      }
+      if (p.status) *p.status = (int)DAD_ERR_TIMEOUT;
+    }
+    __syncthreads();
+  }
+  cluster_barrier_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
 // C[m][n] = sum over splits, in split order, of the partial tiles umma_gemm256_kernel stored
 // ([tile][split][256][256] fp32): four columns per thread, the whole GPU instead of one CTA per tile.
 __global__ void __launch_bounds__(256)
@@ -870,6 +1087,9 @@ static EncodeTiledFn encode_fn() {
 }
 
 bool tmap_encoder_available() { return encode_fn() != nullptr; }
+
+// Whether short dense products may run on CTA pairs (on unless DAD_NO_PAIR_GEMM is set in the environment, for A/B timing).
+static const bool g_pair_gemm = getenv("DAD_NO_PAIR_GEMM") == nullptr;
 
 // bf16 tensor (d0 innermost, contiguous) x d1 x d2 with byte strides s1, s2; box = box0 x box1 x 1,
 // 128-byte swizzle, out-of-range elements read as zero.
@@ -1197,6 +1417,42 @@ static cudaError_t launch_gemm_persist(const CUtensorMap& tmA, const CUtensorMap
 }
 
 
+template <int STAGES>
+static cudaError_t launch_gemm_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                                    const UmmaParams& p, unsigned ctas, cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * (4 * 8192) + 2 * 128 * 128 + 1024;
+  auto kernel = umma_gemm_pair_kernel<STAGES>;
+  cudaError_t err = cudaSuccess;
+  static FirstUse first;
+  if (first.on_this_device()) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) {
+      first.forget();
+      return err;
+    }
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctas, 1, 1);
+  cfg.blockDim = dim3(192, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  const bool timed = g_timing.load(std::memory_order_relaxed);
+  if (timed) timing_mark("gemm_tn_tc", st, true);
+  err = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
+  if (timed) timing_mark("gemm_tn_tc", st, false);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return err;
+}
+
 // C (hx x hy, fp32) <- sum over sites and rows of X^T Y.  tmX: (hx, N, S), tmY: (hy, N, S), boxes 64 x plan.bk.
 // With plan.batch > 1 (and S = 1) the third tensor dimension counts independent products instead: C is batch x hx x hy.
 cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const GemmPlan& g, int64_t hx, int64_t hy,
@@ -1244,6 +1500,14 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
   // Many 128 x 256 tiles of a short contraction over one site per product: the persistent kernel (one CTA per SM, two
   // accumulators).  Its blocks are numbered per product, so a contraction over several sites keeps the per-tile CTAs.
   const int64_t all_tiles = g.tiles * g.batch;
+  // Enough 256 x 256 tiles for every pair of SMs: the pair kernel, which needs a third fewer operand bytes per SM.
+  const int64_t tiles256 = ceil_div(hx, 256) * ceil_div(hy, 256) * g.batch;
+  if (pC && g.bn == 256 && tiles256 >= 74 && g_pair_gemm && (g.batch > 1 || g.k_blocks == g.kb_per_site)) {
+    p.batch_count = g.batch;
+    p.tiles_m = (int)ceil_div(hx, 256);
+    p.tiles_n = (int)ceil_div(hy, 256);
+    return launch_gemm_pair<5>(tmX, tmY, tmC, p, 148u, st);
+  }
   if (pC && g.bn == 256 && all_tiles >= 148 && p.k_blocks <= 8 && (g.batch > 1 || g.k_blocks == g.kb_per_site)) {
     p.batch_count = g.batch;
     return launch_gemm_persist<3>(tmX, tmY, tmC, p, 148u, st);
