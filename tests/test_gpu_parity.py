@@ -420,6 +420,24 @@ def test_many_sites_at_large_rank(oracle, B, iters, dependent_start):
             assert [j for j in range(r) if np.all(g["Q"][s][j] == 0.0)] == [9, r - 1]
 
 
+@pytest.mark.parametrize("S,N,h_in,h_out,r,iters", [
+    (80, 200, 520, 768, 40, 2),     # ragged second row tile, 520 columns = 4 tiles and a sliver
+    (75, 512, 256, 1024, 64, 1),    # whole tiles everywhere
+    (90, 250, 1024, 136, 56, 2),    # a 136-wide operand: one tile and eight columns
+])
+def test_many_sites_above_rank_32(oracle, B, S, N, h_in, h_out, r, iters):
+    """Ranks that pad to 64 on launches of more than one wave of CTAs (the shallow two- and three-stage forms of the thin
+    products, 128-column accumulators), with ragged row and column tiles.  Parity with the oracle on every site at the
+    accuracy the path delivers, and two runs bit for bit."""
+    A, D = wl.decaying_layer(S, N, h_in, h_out, 7300 + N, torch.bfloat16)
+    Q0 = wl.start_block(S, r, h_out, 7300 + N)
+    g1, o = check_layer(oracle, B, A, D, Q0, r, iters, TOL[torch.bfloat16], ortho_tol=1e-3)
+    for s in range(S):
+        assert rel(g1["P"][s].T @ g1["Q"][s], o["P"][s].T @ o["Q"][s]) <= 1e-4
+    g2 = run_gpu_layer(B, A, D, Q0, r, iters)
+    assert np.array_equal(g1["P"], g2["P"]) and np.array_equal(g1["Q"], g2["Q"])
+
+
 def test_edge_shapes(oracle, B):
     # one row, one site, r = 1; r = min(h); zero iterations; strided (non-contiguous) rows and sites
     A, D = wl.gaussian_layer(1, 1, 8, 8, 1)
