@@ -77,6 +77,9 @@ def parse_args():
                          "run reports beside its headline workload")
     ap.add_argument("--sweep-steps", type=int, default=3, help="timed steps of each sweep entry")
     ap.add_argument("--no-check", action="store_true", help="skip the oracle check of one sampled site per workload")
+    ap.add_argument("--reconstruct-per-call", action="store_true",
+                    help="reconstruct after every call instead of once per layer shape and step (one batched call over all "
+                         "of the step's layers of that shape, which fills the GPU's rounds of output tiles)")
     return ap.parse_args()
 
 
@@ -442,6 +445,9 @@ def measure(args, rank, local, world, dev, headline):
                 A, D = wl.decaying_layer(cfg.S * groups, cfg.N, sh.h_in, sh.h_out, seed, cfg.torch_dtype, dev)
             blk.append((A, D, wl.start_block(cfg.S * groups, r, sh.h_out, seed, dev)))
         data.append(blk)
+    # calls of one plan per step: their layers are reconstructed together at the end of the step (one batched call)
+    defer = n_super > 1 and not args.reconstruct_per_call and not args.no_group
+    n_calls = n_super if defer else 1
     plans = {}
     for ui, (sh, groups) in enumerate(units):
         key = (sh.h_in, sh.h_out, groups)
@@ -451,7 +457,7 @@ def measure(args, rank, local, world, dev, headline):
             if cfg.dtype != "f32":
                 terms = args.reconstruct_terms or (1 if cfg.S * r >= 512 else 3)
                 rmath = B.DAD_BF16_1TERM if terms == 1 else B.DAD_BF16
-            plans[key] = B.LayerPlan(A, D, r, iters, groups=groups, reconstruct_math=rmath)
+            plans[key] = B.LayerPlan(A, D, r, iters, groups=groups, reconstruct_math=rmath, calls=n_calls)
     input_bytes = sum(A.numel() * A.element_size() + D.numel() * D.element_size() for blk in data for A, D, _ in blk)
     stream = torch.cuda.current_stream()
     # Calls on different plans are independent (own inputs, workspace and outputs).  Where one call cannot fill the GPU
@@ -471,7 +477,10 @@ def measure(args, rank, local, world, dev, headline):
             for ui, (sh, groups) in enumerate(units):
                 A, D, Q0 = blk[ui]
                 key = (sh.h_in, sh.h_out, groups)
-                plans[key].step(A, D, Q0, lanes[lane_of[key]])
+                plans[key].step(A, D, Q0, lanes[lane_of[key]], call=b if defer else None)
+        if defer:
+            for key, plan in plans.items():
+                plan.finish(lanes[lane_of[key]])
         for sd in side_streams:
             stream.wait_stream(sd)
 
@@ -713,7 +722,9 @@ def measure(args, rank, local, world, dev, headline):
                            "l2": f"inputs larger than L2: {RB} resident input set(s) of {G} block(s), {input_bytes / 1e9:.2f} GB, cycled",
                            "calls": ("one call per layer" if args.no_group else
                                      f"same-shape layers of {G} consecutive block(s) stacked as extra slices of one call: " +
-                                     ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units)),
+                                     ", ".join(f"{g}x {sh.h_in}->{sh.h_out}" for sh, g in units) +
+                                     (f"; the {n_super} calls of a shape per step compress and gather, one batched "
+                                      "reconstruction per shape ends the step" if defer else "")),
                            "launch": ("CUDA graph replay" if args.cuda_graph else "stream launches") +
                                      ("" if n_streams == 1 else
                                       f", the step's independent calls dealt over {n_streams} streams"),

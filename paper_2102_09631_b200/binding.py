@@ -377,26 +377,38 @@ class LayerPlan:
     `groups` > 1 stacks that many layers of the same shape in one plan: A and D then hold
     groups * S slices (layer g owns slices g*S .. g*S+S-1), the power iterations of all of them run
     in the same launches (slices are independent), and each layer is reconstructed from its own rows
-    of the stacks (one batched call); `grad` is then groups x h_in x h_out."""
+    of the stacks (one batched call); `grad` is then groups x h_in x h_out.
+
+    `calls` > 1 keeps the factors and stacks of that many calls of the plan side by side: `step(..., call=c)`
+    compresses and gathers into slot c without reconstructing, and `finish()` reconstructs the layers of all
+    slots in ONE batched call (`grads_all`: calls * groups x h_in x h_out).  The reconstruction of a handful of
+    layers is a few tens of microseconds of work that does not fill the GPU's last round of tiles; a step's worth
+    of a shape does."""
 
     def __init__(self, A: torch.Tensor, D: torch.Tensor, r: int, iters: int, zero_copy_gather: bool = False,
-                 groups: int = 1, reconstruct_math: Optional[int] = None):
+                 groups: int = 1, reconstruct_math: Optional[int] = None, calls: int = 1):
         self.layer = make_layer(A, D)
         L = self.layer
         if groups < 1 or L.S % groups:
             raise ValueError("the slice count must be a multiple of `groups`")
-        self.groups, self.sites = groups, L.S // groups
+        if calls < 1:
+            raise ValueError("`calls` must be at least 1")
+        self.groups, self.sites, self.calls = groups, L.S // groups, calls
         dev = A.device
         self.r, self.iters = r, iters
-        self.P = torch.empty(L.S, r, L.h_in, device=dev, dtype=torch.float32)
-        self.Q = torch.empty(L.S, r, L.h_out, device=dev, dtype=torch.float32)
-        self.sigma = torch.empty(L.S, r, device=dev, dtype=torch.float32)
+        self.P_all = torch.empty(calls, L.S, r, L.h_in, device=dev, dtype=torch.float32)
+        self.Q_all = torch.empty(calls, L.S, r, L.h_out, device=dev, dtype=torch.float32)
+        self.sigma_all = torch.empty(calls, L.S, r, device=dev, dtype=torch.float32)
         if zero_copy_gather:
-            self.Pcat, self.Qcat = self.P.view(L.S * r, L.h_in), self.Q.view(L.S * r, L.h_out)
+            self.Pcat_all, self.Qcat_all = self.P_all.view(calls, L.S * r, L.h_in), self.Q_all.view(calls, L.S * r, L.h_out)
         else:
-            self.Pcat = torch.empty(L.S * r, L.h_in, device=dev, dtype=torch.float32)
-            self.Qcat = torch.empty(L.S * r, L.h_out, device=dev, dtype=torch.float32)
-        self.grads = torch.empty(groups, L.h_in, L.h_out, device=dev, dtype=torch.float32)
+            self.Pcat_all = torch.empty(calls, L.S * r, L.h_in, device=dev, dtype=torch.float32)
+            self.Qcat_all = torch.empty(calls, L.S * r, L.h_out, device=dev, dtype=torch.float32)
+        self.grads_all = torch.empty(calls * groups, L.h_in, L.h_out, device=dev, dtype=torch.float32)
+        # slot 0 under the names a plan of one call has always had
+        self.P, self.Q, self.sigma = self.P_all[0], self.Q_all[0], self.sigma_all[0]
+        self.Pcat, self.Qcat = self.Pcat_all[0], self.Qcat_all[0]
+        self.grads = self.grads_all[:groups]
         self.grad = self.grads[0] if groups == 1 else self.grads
         # reconstruction arithmetic: that of the inputs (fp32 FMA / three-term bf16) unless the caller picks one
         self.math = L.dtype if reconstruct_math is None else reconstruct_math
@@ -406,12 +418,29 @@ class LayerPlan:
         self.K = self.sites * r
         self.ws = new_workspace(max(nws, dad_reconstruct_batched_workspace_bytes(L.h_in, L.h_out, self.K, groups,
                                                                                  self.math)), dev)
+        self.ws_all = None
+        if calls > 1:
+            self.ws_all = new_workspace(max(256, dad_reconstruct_batched_workspace_bytes(L.h_in, L.h_out, self.K,
+                                                                                          calls * groups, self.math)), dev)
         self.bytes_tx = bytes_array(L.S)
 
-    def step(self, A, D, Q0, stream=None):
+    def step(self, A, D, Q0, stream=None, call: Optional[int] = None):
         L = self.layer
-        dad_rank_compress(L, A, D, self.r, self.iters, Q0, self.P, self.Q, self.sigma, self.ws, stream)
-        dad_gather_factors(L, self.r, self.P, self.Q, self.Pcat, self.Qcat, self.bytes_tx, stream)
-        dad_reconstruct_batched(L.h_in, L.h_out, self.K, self.groups, self.Pcat, self.Qcat, self.grads, self.math,
-                                self.ws, stream)
-        return self.grad
+        if call is None:
+            dad_rank_compress(L, A, D, self.r, self.iters, Q0, self.P, self.Q, self.sigma, self.ws, stream)
+            dad_gather_factors(L, self.r, self.P, self.Q, self.Pcat, self.Qcat, self.bytes_tx, stream)
+            dad_reconstruct_batched(L.h_in, L.h_out, self.K, self.groups, self.Pcat, self.Qcat, self.grads, self.math,
+                                    self.ws, stream)
+            return self.grad
+        P, Q = self.P_all[call], self.Q_all[call]
+        dad_rank_compress(L, A, D, self.r, self.iters, Q0, P, Q, self.sigma_all[call], self.ws, stream)
+        dad_gather_factors(L, self.r, P, Q, self.Pcat_all[call], self.Qcat_all[call], self.bytes_tx, stream)
+        return None
+
+    def finish(self, stream=None):
+        """Reconstructs the layers of every slot filled by `step(..., call=c)` in one batched call."""
+        L = self.layer
+        ws = self.ws_all if self.ws_all is not None else self.ws
+        dad_reconstruct_batched(L.h_in, L.h_out, self.K, self.calls * self.groups, self.Pcat_all, self.Qcat_all,
+                                self.grads_all, self.math, ws, stream)
+        return self.grads_all

@@ -664,6 +664,32 @@ def test_stacked_layers_match_separate_calls(oracle, B):
     assert list(plan.bytes_tx) == [oracle.bytes_rank(r, h_in, h_out)] * (S * groups)
 
 
+def test_reconstruction_deferred_to_one_batched_call(oracle, B):
+    """A plan of several calls (LayerPlan(calls=3)): every call compresses and gathers into its own slot, finish()
+    reconstructs the layers of all slots in one batched call.  Bit for bit what per-call plans give, and one layer
+    against the oracle."""
+    dev = torch.device("cuda:0")
+    S, N, h_in, h_out, r, iters, groups, calls = 3, 260, 512, 768, 8, 2, 2, 3
+    sets = []
+    for c in range(calls):
+        A, D = wl.decaying_layer(S * groups, N, h_in, h_out, 8800 + c, torch.bfloat16, device=dev)
+        sets.append((A, D, wl.start_block(S * groups, r, h_out, 8800 + c, dev)))
+    plan = B.LayerPlan(*sets[0][:2], r, iters, groups=groups, calls=calls)
+    for c, (A, D, Q0) in enumerate(sets):
+        plan.step(A, D, Q0, call=c)
+    grads = plan.finish()
+    B.dad_check(plan.ws)
+    B.dad_check(plan.ws_all)
+    single = B.LayerPlan(*sets[0][:2], r, iters, groups=groups)
+    for c, (A, D, Q0) in enumerate(sets):
+        g = single.step(A, D, Q0)
+        assert torch.equal(g, grads[c * groups:(c + 1) * groups])
+        assert torch.equal(single.P, plan.P_all[c]) and torch.equal(single.Q, plan.Q_all[c])
+    A, D, Q0 = sets[1]
+    o = oracle.rank_dad_layer(A[S:2 * S].cpu(), D[S:2 * S].cpu(), Q0[S:2 * S].cpu(), iters)   # call 1, second layer
+    assert rel(grads[1 * groups + 1].double().cpu().numpy(), o["grad"]) <= ACCURACY_BAR
+
+
 def test_host_entry_point_matches_device_path_and_oracle(oracle, B):
     """dad_rank_dad_host: inputs in (pinned) host memory, gradient back in host memory; same result as the
     three device calls, bit for bit, for dense and for strided host layouts."""
