@@ -599,26 +599,33 @@ def measure(args, rank, local, world, dev, headline):
         flops_total, ms_total = 0.0, 0.0
         for ui, (sh, groups) in enumerate(units):
             A, D, _ = data[0][ui]
-            A1, D1 = A[:cfg.S], D[:cfg.S]          # one layer's slices
+            # Layers of one shape whose single gradient is too few output tiles for the GPU share a launch
+            # (dad_full_grad_grouped): as many of the call's stacked layers as bring the tiles of 256 x 256 to about 64.
+            tiles1 = -(-sh.h_in // 256) * -(-sh.h_out // 256)
+            gg = 1
+            while gg * 2 <= groups and groups % (gg * 2) == 0 and tiles1 * gg * 2 <= 64:
+                gg *= 2
+            A1, D1 = A[:cfg.S * gg], D[:cfg.S * gg]          # gg layers' slices
             L1 = B.make_layer(A1, D1)
-            g = torch.empty(sh.h_in, sh.h_out, device=dev, dtype=torch.float32)
-            ws = B.new_workspace(B.dad_workspace_bytes(L1, 1, 0), dev)
+            g = torch.empty(gg, sh.h_in, sh.h_out, device=dev, dtype=torch.float32)
+            ws = B.new_workspace(max(256, B.dad_full_grad_grouped_workspace_bytes(L1, gg)), dev)
             for _ in range(2):
-                B.dad_full_grad(L1, A1, D1, g, None, ws, stream)
+                B.dad_full_grad_grouped(L1, gg, A1, D1, g, None, ws, stream)
             f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             reps = 5
             torch.cuda.synchronize()
             f0.record(stream)
             for _ in range(reps):
-                B.dad_full_grad(L1, A1, D1, g, None, ws, stream)
+                B.dad_full_grad_grouped(L1, gg, A1, D1, g, None, ws, stream)
             f1.record(stream)
             torch.cuda.synchronize()
             B.dad_check(ws)
-            t_ms = f0.elapsed_time(f1) / reps
+            t_ms = f0.elapsed_time(f1) / reps / gg          # per layer
             fl = 2.0 * cfg.S * cfg.N * sh.h_in * sh.h_out
             flops_total += fl * sh.count
             ms_total += t_ms * sh.count
-            rows.append({"layer": f"{sh.h_in}->{sh.h_out}", "us": t_ms * 1e3, "tflops": fl / (t_ms * 1e-3) / 1e12})
+            rows.append({"layer": f"{sh.h_in}->{sh.h_out}", "us": t_ms * 1e3, "tflops": fl / (t_ms * 1e-3) / 1e12,
+                         "layers_per_call": gg})
         tf = flops_total / (ms_total * 1e-3) / 1e12
         full_grad = {"bound": "tensor" if cfg.dtype == "bf16" else "alu", "achieved": tf, "peak": peaks["bf16_tflops"],
                      "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",

@@ -114,6 +114,22 @@ dad_status dad_full_grad(const dad_layer* layer, const void* A, const void* D, f
                          uint64_t* bytes_tx, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The same gradient (Sec. 3.2; Eq. "local_grad") for `groups` layers of one shape in one call: `layer` describes
+ * groups * S' slices, layer g owning slices g*S' .. g*S'+S'-1 (S' = layer->S / groups, which must divide), and
+ *     grads[g][a][b] = sum over the slices s of layer g and the rows n of  A_s[n][a] * D_s[n][b].
+ * One launch then serves all of them where a single layer's output tiles would leave part of the GPU idle (a
+ * 1024 x 1024 gradient is 16 tiles of 256 x 256 for 148 SMs).  Arguments as dad_full_grad, with
+ *   grads    DEVICE, groups x h_in x h_out fp32, contiguous, 16-byte aligned
+ *   bytes_tx HOST, layer->S entries, or NULL
+ *   ws       DEVICE scratch of ws_bytes >= dad_full_grad_grouped_workspace_bytes(layer, groups)
+ * Shapes the large-tile tensor-core kernel does not take are computed one layer after the other.
+ * DAD_ERR_SHAPE if groups < 1 or does not divide layer->S.
+ */
+size_t dad_full_grad_grouped_workspace_bytes(const dad_layer* layer, int groups);
+dad_status dad_full_grad_grouped(const dad_layer* layer, int groups, const void* A, const void* D, float* grads,
+                                 uint64_t* bytes_tx, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Structured power iterations, all r vectors of a site advanced together (Algorithm 2;
  * Eq. "nabla_iter" evaluated through A and D as in Eq. "reduced_iter", never forming the
  * h_in x h_out gradient; the peel term of Eq. "peel" realised as orthonormalisation of the

@@ -24,6 +24,7 @@ STATUS_NAMES = ["DAD_OK", "DAD_ERR_NULL", "DAD_ERR_SHAPE", "DAD_ERR_DTYPE", "DAD
 
 # every symbol include/dad.h declares
 EXPORTS = ["dad_bytes_dad", "dad_bytes_rank", "dad_bytes_dsgd", "dad_workspace_bytes", "dad_full_grad",
+           "dad_full_grad_grouped_workspace_bytes", "dad_full_grad_grouped",
            "dad_rank_compress", "dad_gather_factors", "dad_reconstruct_workspace_bytes", "dad_reconstruct",
            "dad_reconstruct_batched_workspace_bytes", "dad_reconstruct_batched",
            "dad_reconstruct_static", "dad_aggregate_workspace_bytes", "dad_aggregate_compress", "dad_effective_rank",
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.dad_workspace_bytes.restype = ctypes.c_size_t
         L.dad_full_grad.argtypes = [lp, vp, vp, vp, u64p, vp, ctypes.c_size_t, vp]
         L.dad_full_grad.restype = ctypes.c_int
+        L.dad_full_grad_grouped_workspace_bytes.argtypes = [lp, ctypes.c_int]
+        L.dad_full_grad_grouped_workspace_bytes.restype = ctypes.c_size_t
+        L.dad_full_grad_grouped.argtypes = [lp, ctypes.c_int, vp, vp, vp, u64p, vp, ctypes.c_size_t, vp]
+        L.dad_full_grad_grouped.restype = ctypes.c_int
         L.dad_rank_compress.argtypes = [lp, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.dad_rank_compress.restype = ctypes.c_int
         L.dad_gather_factors.argtypes = [lp, ctypes.c_int, vp, vp, vp, vp, u64p, vp]
@@ -221,6 +226,17 @@ def dad_full_grad(layer: dad_layer, A, D, grad, bytes_tx=None, ws=None, stream=N
     st = lib().dad_full_grad(ctypes.byref(layer), _ptr(A), _ptr(D), _ptr(grad), bytes_tx, _ptr(ws),
                              ws.numel() if ws is not None else 0, _stream(stream))
     _check(st, "dad_full_grad")
+
+
+def dad_full_grad_grouped_workspace_bytes(layer: dad_layer, groups: int) -> int:
+    return int(lib().dad_full_grad_grouped_workspace_bytes(ctypes.byref(layer), groups))
+
+
+def dad_full_grad_grouped(layer: dad_layer, groups: int, A, D, grads, bytes_tx=None, ws=None, stream=None):
+    """grads (groups x h_in x h_out fp32) <- the dAD gradients of `groups` layers stacked as slices of A and D."""
+    st = lib().dad_full_grad_grouped(ctypes.byref(layer), groups, _ptr(A), _ptr(D), _ptr(grads), bytes_tx, _ptr(ws),
+                                     ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "dad_full_grad_grouped")
 
 
 def dad_rank_compress(layer: dad_layer, A, D, r: int, iters: int, Q0, P, Q, sigma, ws, stream=None):

@@ -124,13 +124,13 @@ CompressWs compress_ws_layout(const dad_layer& L, int r, bool f64, bool tc, int 
   return w;
 }
 
-GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands, int batch) {
+GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands, int batch, int products) {
   GemmWs w;
   memset(&w, 0, sizeof(w));
   size_t off = 0;
   w.status = off;
   off += 256;
-  const GemmPlan g = umma_gemm_plan(hx, hy, S, N, batch);
+  const GemmPlan g = umma_gemm_plan(hx, hy, S, N, batch, products);
   const size_t tiles = (size_t)g.tiles * (size_t)batch;
   w.n_counters = tiles;
   w.counters = off;
@@ -288,13 +288,14 @@ static cudaError_t run_compress_tc(const dad_layer& L, const void* A, const void
 
 static cudaError_t run_gemm_tc(const void* X, int64_t ldX, int64_t strideX, const void* Y, int64_t ldY, int64_t strideY,
                                int S, int64_t N, int64_t hx, int64_t hy, float* C, char* ws, const GemmWs& w,
-                               cudaStream_t st, int batch = 1) {
+                               cudaStream_t st, int batch = 1, int products = 1) {
   // the second status slot (byte 4) belongs to the dense products; the first keeps what a compress call reported
   cudaError_t err = cudaMemsetAsync(ws + w.status + 4, 0, w.counters + w.n_counters * sizeof(unsigned) - w.status - 4, st);
   if (err != cudaSuccess) return err;
   CUtensorMap tmX, tmY;
-  const GemmPlan g = umma_gemm_plan(hx, hy, S, N, batch);
-  const uint64_t d2 = batch > 1 ? (uint64_t)batch : (uint64_t)S;  // third dimension: sites of one product, or products
+  const GemmPlan g = umma_gemm_plan(hx, hy, S, N, batch, products);
+  // third dimension: the sites of one product (of `products` products of S sites each), or one-site products
+  const uint64_t d2 = batch > 1 ? (uint64_t)batch : (uint64_t)S * (uint64_t)products;
   if (!make_tmap_bf16_3d(&tmX, X, hx, N, d2, (uint64_t)ldX * 2, (uint64_t)strideX * 2, 64, (uint32_t)g.bk) ||
       !make_tmap_bf16_3d(&tmY, Y, hy, N, d2, (uint64_t)ldY * 2, (uint64_t)strideY * 2, 64, (uint32_t)g.bk))
     return cudaErrorInvalidValue;
@@ -368,6 +369,59 @@ dad_status dad_full_grad(const dad_layer* layer, const void* A, const void* D, f
   if (err != cudaSuccess) return DAD_ERR_CUDA;
   if (bytes_tx)
     for (int s = 0; s < L->S; ++s) bytes_tx[s] = dad_bytes_dad(L);
+  return DAD_OK;
+}
+
+// Whether `groups` gradients of this shape run as one launch of the 256 x 256 kernel (else one call per layer).
+static bool full_grad_grouped_tc(const dad_layer& L, int groups) {
+  if (!tc_eligible(L)) return false;
+  const GemmPlan g = umma_gemm_plan(L.h_in, L.h_out, L.S / groups, L.N, 1, groups);
+  return g.bm == 256;
+}
+
+size_t dad_full_grad_grouped_workspace_bytes(const dad_layer* layer, int groups) {
+  if (validate_layer(layer) != DAD_OK || groups < 1 || layer->S % groups != 0) return 0;
+  const dad_layer L = normalised(*layer);
+  if (full_grad_grouped_tc(L, groups)) return gemm_ws_layout(L.h_in, L.h_out, L.S / groups, L.N, false, 1, groups).total;
+  dad_layer one = L;
+  one.S = L.S / groups;
+  return dad_workspace_bytes(&one, 1, 0);
+}
+
+dad_status dad_full_grad_grouped(const dad_layer* layer, int groups, const void* A, const void* D, float* grads,
+                                 uint64_t* bytes_tx, void* ws, size_t ws_bytes, void* cuda_stream) {
+  dad_status vs = validate_layer(layer);
+  if (vs != DAD_OK) return vs;
+  if (groups < 1 || layer->S % groups != 0) return DAD_ERR_SHAPE;
+  const dad_layer L = normalised(*layer);
+  if (!A || !D || !grads) return DAD_ERR_NULL;
+  if (!aligned(A, 16) || !aligned(D, 16) || !aligned(grads, 16)) return DAD_ERR_ALIGN;
+  const int Sg = L.S / groups;
+  if (groups > 1 && full_grad_grouped_tc(L, groups)) {
+    const GemmWs w = gemm_ws_layout(L.h_in, L.h_out, Sg, L.N, false, 1, groups);
+    if (!ws) return DAD_ERR_NULL;
+    if (!aligned(ws, 256)) return DAD_ERR_ALIGN;
+    if (ws_bytes < w.total) return DAD_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const BoundsRange ranges[] = {{A, operand_bytes(L, true)}, {D, operand_bytes(L, false)},
+                                  {grads, sizeof(float) * (size_t)groups * L.h_in * L.h_out}, {ws, ws_bytes}};
+    if (bounds_register(ranges, 4, st) != cudaSuccess) return DAD_ERR_CUDA;
+    const cudaError_t err = run_gemm_tc(A, L.ldA, L.strideA, D, L.ldD, L.strideD, Sg, L.N, L.h_in, L.h_out, grads, (char*)ws, w,
+                                        st, 1, groups);
+    if (err != cudaSuccess) return DAD_ERR_CUDA;
+  } else {
+    dad_layer one = L;  // one call per layer: its sites are slices g * Sg ... of the stacked buffers
+    one.S = Sg;
+    const size_t e = L.dtype == DAD_F32 ? 4 : 2;
+    for (int g = 0; g < groups; ++g) {
+      const dad_status st1 = dad_full_grad(&one, (const char*)A + e * (size_t)g * Sg * L.strideA,
+                                           (const char*)D + e * (size_t)g * Sg * L.strideD,
+                                           grads + (size_t)g * L.h_in * L.h_out, nullptr, ws, ws_bytes, cuda_stream);
+      if (st1 != DAD_OK) return st1;
+    }
+  }
+  if (bytes_tx)
+    for (int s = 0; s < L.S; ++s) bytes_tx[s] = dad_bytes_dad(&L);
   return DAD_OK;
 }
 

@@ -108,7 +108,7 @@ cudaError_t fused_compress(const dad_layer& L, const void* A, const void* D, int
 struct GemmWs {
   size_t status, counters, n_counters, partial, Xb, Yb, total;  // Xb/Yb: bf16 copies of fp32 operands
 };
-GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands, int batch = 1);
+GemmWs gemm_ws_layout(int64_t hx, int64_t hy, int S, int64_t N, bool convert_operands, int batch = 1, int products = 1);
 
 // Whether the tensor-core kernels take this layer: bf16, all extents and strides multiples of 8
 // elements (TMA wants 16-byte strides), and the driver's tensor-map encoder is available.
@@ -179,12 +179,13 @@ int umma_cols_acc_splits(int S, int64_t N, int64_t h);
 // bk contraction rows (the row count of the operands' TMA boxes), `splits` CTAs share a tile's contraction.
 struct GemmPlan {
   int bm, bn, bk, splits, batch;
+  int products;                          // 256 x 256 tiles: products of S sites each that share the launch (tiles counts all)
   int rem_ctas;                          // 256 x 256 tiles: CTAs that take the tail of every tile's contraction
   int64_t tiles, k_blocks, kb_per_site;  // tiles: per batch entry
   int64_t kb_per_split;                  // blocks of each of the `splits` equal parts
 };
 // batch > 1: that many independent products of one site each (S must be 1) in one launch.
-GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch);
+GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch, int products = 1);
 cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S, int64_t N, int64_t h, int r,
                           __nv_bfloat16* yt_planes, int64_t ld_planes, int* status, cudaStream_t st);
 cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S, int64_t N, int64_t h, int r, float* out,

@@ -55,7 +55,8 @@ struct UmmaParams {
   float* partial;    // split partial tiles [tile][split][128][BN]
   unsigned* counters;
   int* status;
-  int batch_count;      // persistent dense-product kernel: products in the launch (its grid is one-dimensional)
+  int batch_count;      // persistent dense-product kernels and the 256 x 256 kernel: products in the launch
+  int sites_per_product;  // 256 x 256 kernel: sites of each product (product g reads sites g * sites_per_product ...)
   int tma_store;        // EPI_C without a split contraction: the tile leaves through shared memory and TMA stores (tmC)
   uint32_t wait_limit;  // polls a bounded wait may take; 0 = kWaitLimit
   int expect_extra_kb;  // self-test only: the MMA role waits for this many blocks more than the producer loads
@@ -429,13 +430,14 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // first splits * kb_per_split blocks of the contraction (m fastest, so neighbours share a B panel at the same k).
   // The rem_ctas CTAs after them take what is left of the contraction, the same block range for every tile, each for
   // the tiles t = j, j + rem_ctas, ... one after the other: they fill the SMs that tiles * splits leaves empty.
-  const int n_tiles = p.tiles_m * p.tiles_n;
+  const int tiles_per_product = p.tiles_m * p.tiles_n;
+  const int n_tiles = tiles_per_product * p.batch_count;  // several products of one shape share a launch
   const int n_main = n_tiles * p.splits;
   const bool is_rem = (int)blockIdx.x >= n_main;
   const int rem_j = (int)blockIdx.x - n_main;
   const int slots = p.splits + (p.rem_ctas > 0 ? 1 : 0);  // partial tiles per output tile
   struct Item {
-    int m0, n0, kb0, kb1, slot;
+    int m0, n0, kb0, kb1, slot, product;
     int64_t tile_lin;
   };
   auto item_at = [&](int it, Item& w) -> bool {
@@ -456,11 +458,13 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       w.kb1 = p.k_blocks;
     }
     if (w.kb1 < w.kb0) w.kb1 = w.kb0;
-    const int m_tile = tile % p.tiles_m, n_tile = tile / p.tiles_m;
+    w.product = tile / tiles_per_product;
+    const int rem = tile - w.product * tiles_per_product;
+    const int m_tile = rem % p.tiles_m, n_tile = rem / p.tiles_m;
     w.m0 = m_tile * 256;
     w.n0 = n_tile * 256;
     w.slot = split;
-    w.tile_lin = (int64_t)m_tile * p.tiles_n + n_tile;
+    w.tile_lin = (int64_t)w.product * tiles_per_product + (int64_t)m_tile * p.tiles_n + n_tile;
     return true;
   };
 
@@ -508,7 +512,7 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
           uint8_t* a_dst = smem + (size_t)stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_BYTES;
-          const int bz = kb / p.kb_per_site;
+          const int bz = w.product * p.sites_per_product + kb / p.kb_per_site;
           const int kcoord = (kb % p.kb_per_site) * BK;
 #pragma unroll
           for (int c = 0; c < 4; ++c) tma_load_3d(a_dst + c * CHUNK, &tmA, &full_bar[stage], w.m0 + c * 64, kcoord, bz);
@@ -582,7 +586,7 @@ umma_gemm256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else {
           const int64_t gm = (int64_t)w.m0 + half * 128 + row;
           if (gm < p.m_extent) {
-            float* dst = p.out_f32 + gm * p.ld_out + w.n0 + col;
+            float* dst = p.out_f32 + (int64_t)w.product * p.out_batch_stride + gm * p.ld_out + w.n0 + col;
             if (w.n0 + col + 16 <= p.n_extent && (p.ld_out & 3) == 0) {
 #pragma unroll
               for (int i = 0; i < 4; ++i)
@@ -1053,6 +1057,9 @@ gemm256_reduce_kernel(const float* __restrict__ partial, int splits, int m_exten
   const int n4 = n_extent / 4;  // n_extent is a multiple of 8 on this path
   const int tiles_n = (n_extent + 255) / 256;
   const int64_t total = (int64_t)m_extent * n4;
+  // one product per blockIdx.y: its partial tiles and its C follow the previous product's
+  partial += (int64_t)blockIdx.y * ((m_extent + 255) / 256) * tiles_n * splits * (int64_t)(256 * 256);
+  C += (int64_t)blockIdx.y * m_extent * n_extent;
   for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     const int m = (int)(idx / n4), n = (int)(idx % n4) * 4;
     const int64_t tile = (int64_t)(m / 256) * tiles_n + n / 256;
@@ -1303,15 +1310,16 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
 // the 256 x 256 two-accumulator kernel; everything else 128 x BN tiles, BN = 256 where the output is wide
 // enough (a 128 x 128 x 16 MMA needs 128 B/clk of operands from shared memory, a 128 x 256 x 16 one
 // 96 B/clk).  Splits of the contraction fill the 148 SMs when the tiles alone do not.
-GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch) {
+GemmPlan umma_gemm_plan(int64_t hx, int64_t hy, int S, int64_t N, int batch, int products) {
   GemmPlan g;
+  g.products = products;
   const bool big = batch == 1 && hx >= 256 && hy >= 256 && N * S >= kGemm256MinRows;
   int64_t min_blocks;
   if (big) {
     g.bm = 256;
     g.bn = 256;
     g.bk = kGemm256BK;
-    g.tiles = ceil_div(hx, 256) * ceil_div(hy, 256);
+    g.tiles = ceil_div(hx, 256) * ceil_div(hy, 256) * products;  // of all the products of the launch
     min_blocks = 512 / g.bk;
   } else {
     g.bm = 128;
@@ -1475,14 +1483,18 @@ cudaError_t umma_gemm_tn(const CUtensorMap& tmX, const CUtensorMap& tmY, const G
   p.status = status;
   dim3 grid((unsigned)ceil_div(hx, g.bm), (unsigned)(ceil_div(hy, g.bn) * g.splits), (unsigned)g.batch);
   if (g.bm == 256) {
+    p.batch_count = g.products;
+    p.sites_per_product = (int)(g.k_blocks / g.kb_per_site);
     const int slots = g.splits + (g.rem_ctas > 0 ? 1 : 0);
     const dim3 grid1((unsigned)(g.tiles * g.splits + g.rem_ctas), 1, 1);
     cudaError_t err = launch_gemm256<kGemm256BK, kGemm256Stages>(tmX, tmY, p, grid1, st);
     if (err != cudaSuccess || slots == 1) return err;
     const int64_t quads = hx * hy / 4;
     unsigned blocks = (unsigned)(quads / 256 < 148 * 8 ? ceil_div(quads, 256) : 148 * 8);
-    DAD_LAUNCH(err, "gemm_tn_reduce", gemm256_reduce_kernel, blocks, 256, 0, st, (const float*)partial, slots, (int)hx,
-               (int)hy, C);
+    blocks = (blocks + g.products - 1) / g.products;
+    if (blocks < 1) blocks = 1;
+    DAD_LAUNCH(err, "gemm_tn_reduce", gemm256_reduce_kernel, dim3(blocks, (unsigned)g.products, 1), 256, 0, st,
+               (const float*)partial, slots, (int)hx, (int)hy, C);
     return err;
   }
   // Short contractions (the reconstruction: 3 S r rows) spend as long in the epilogue -- 128 KB of fp32 per tile -- as in

@@ -312,6 +312,47 @@ def test_full_grad_long_contraction(oracle, B, S, N, h_in, h_out):
     assert rel(grads[0].double().numpy(), oracle.full_grad(A, D)) <= 1e-4
 
 
+@pytest.mark.parametrize("S,groups,N,h_in,h_out,dtype", [
+    (8, 4, 2048, 1024, 1024, torch.bfloat16),    # four 1024 x 1024 gradients: 64 tiles, split contraction, remainder CTAs
+    (6, 3, 1500, 520, 264, torch.bfloat16),      # ragged tiles, rows no multiple of a stage, three products
+    (4, 2, 300, 128, 96, torch.bfloat16),        # too small for the large tiles: one call per layer inside
+    (4, 2, 64, 40, 24, torch.float32),           # fp32 inputs: the FMA kernel, one call per layer inside
+])
+def test_full_grad_of_several_stacked_layers_in_one_call(oracle, B, S, groups, N, h_in, h_out, dtype):
+    """dad_full_grad_grouped: layer g owns slices g*S' .. of A and D; every gradient against the oracle on its own
+    slices, against dad_full_grad on the same slices, two runs bit for bit, guard bands around the output intact."""
+    dev = torch.device("cuda:0")
+    A, D = wl.gaussian_layer(S, N, h_in, h_out, 515 + N, dtype, dev)
+    L = B.make_layer(A, D)
+    ws = B.new_workspace(max(256, B.dad_full_grad_grouped_workspace_bytes(L, groups)), dev)
+    Sg = S // groups
+    outs = []
+    for _ in range(2):
+        guard = Guarded(groups * h_in * h_out * 4, dev)
+        grads = guard.view((groups, h_in, h_out), torch.float32)
+        tx = B.bytes_array(S)
+        B.dad_full_grad_grouped(L, groups, A, D, grads, tx, ws)
+        B.dad_check(ws)
+        torch.cuda.synchronize()
+        assert guard.intact()
+        outs.append(grads.clone())
+    assert torch.equal(outs[0], outs[1])
+    assert list(tx) == [oracle.bytes_dad(N, h_in, h_out, A.element_size())] * S
+    tol = 1e-4 if dtype == torch.bfloat16 else 1e-5
+    for g in range(groups):
+        sl = slice(g * Sg, (g + 1) * Sg)
+        ref = oracle.full_grad(A[sl].cpu(), D[sl].cpu())
+        assert rel(outs[0][g].double().cpu().numpy(), ref) <= tol, g
+        L1 = B.make_layer(A[sl], D[sl])
+        ws1 = B.new_workspace(max(256, B.dad_workspace_bytes(L1, 1, 0)), dev)
+        one = torch.empty(h_in, h_out, device=dev)
+        B.dad_full_grad(L1, A[sl], D[sl], one, None, ws1)
+        B.dad_check(ws1)
+        assert rel(outs[0][g].double().cpu().numpy(), one.double().cpu().numpy()) <= tol
+    with pytest.raises(Exception):
+        B.dad_full_grad_grouped(L, S + 1, A, D, outs[0], None, ws)     # does not divide the slices
+
+
 @pytest.mark.parametrize("h_in,h_out", [(512, 5120), (520, 5000)])   # whole tiles; ragged last tile row and column
 def test_full_grad_with_remainder_ctas(oracle, B, h_in, h_out):
     """40 tiles of 256 x 256 in 3 splits leave 28 SMs without a CTA; those take the tail of every tile's contraction,
