@@ -1229,17 +1229,17 @@ cudaError_t umma_rows_dot(const CUtensorMap& tmX, const CUtensorMap& tmF, int S,
   p.plane_rows = umma_rank_pad(r);
   p.status = status;
   dim3 grid((unsigned)ceil_div(N, 128), 1, (unsigned)S);
-  // A launch of at most one or two CTAs per SM has no neighbours to cover a CTA's load latency: there the CTA keeps
-  // eight (or four) stages in flight itself (64 CTAs streaming 2048-wide rows: 17.4 us with two stages).
+  // A launch of at most two CTAs per SM has few neighbours to cover a CTA's load latency: there the CTA keeps four
+  // stages in flight itself (64 CTAs streaming 2048-wide rows: 17.4 us with two stages, 15 with four, 14.2 with eight).
+  // Not eight: a 161 KB CTA takes its SM for itself, and such launches come from calls small enough to be run side by
+  // side on several streams (one encoder layer, three calls on three streams: 0.369 ms per step with eight stages,
+  // 0.359 with five, 0.354 with four, 0.365-0.388 with three).
   const int64_t ctas = (int64_t)grid.x * grid.z;
   switch (umma_rank_pad(r)) {
     case 16:
-      if (ctas <= 148) return launch_umma<16, false, false, 2, EPI_YT, 8>(tmX, tmF, p, grid, "rows_dot_tc", st);
       if (ctas <= 2 * 148) return launch_umma<16, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
       return launch_umma<16, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
-    case 32:
-      if (ctas <= 148) return launch_umma<32, false, false, 2, EPI_YT, 8>(tmX, tmF, p, grid, "rows_dot_tc", st);
-      return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
+    case 32: return launch_umma<32, false, false, 2, EPI_YT, 4>(tmX, tmF, p, grid, "rows_dot_tc", st);
     default:
       if (ctas <= 148) return launch_umma<64, false, false, 2, EPI_YT, 6>(tmX, tmF, p, grid, "rows_dot_tc", st);
       return launch_umma<64, false, false, 2, EPI_YT, 2>(tmX, tmF, p, grid, "rows_dot_tc", st);
@@ -1296,10 +1296,15 @@ cudaError_t umma_cols_acc(const CUtensorMap& tmX, const CUtensorMap& tmYt, int S
   switch (umma_rank_pad(r)) {
     // r <= 16: when the launch has CTAs for many waves, five shallow CTAs per SM stream better than two deep ones, as
     // in rows_dot (2 / 3 / 4 / 5 stages: 30.8 / 31.0 / 31.2 / 31.5 ms per benchmark step of 2048-CTA launches); with
-    // fewer CTAs the 740 slots of the shallow form leave a nearly empty last wave (768 CTAs: 9.2 -> 10.7 ms).
+    // fewer CTAs the 740 slots of the shallow form leave a nearly empty last wave (768 CTAs: 9.2 -> 10.7 ms).  CTAs of
+    // at most 16 blocks -- the launches of small calls, which run side by side with other calls' kernels on several
+    // streams -- take three stages: they never fill five, and a smaller CTA leaves more of the SM to the neighbours
+    // (one encoder layer, three calls on three streams: 0.354 -> 0.344 ms per step; 0.363 with two stages).  Long
+    // CTAs that have an SM to themselves keep five (128 CTAs of 64 blocks: 48.2 ms per step with three, 41.4 with five).
     case 16:
       if ((int64_t)grid.x * grid.y * grid.z >= 12 * 148)
         return launch_umma<16, true, false, 2, EPI_Z, 2>(tmX, tmYt, p, grid, "cols_acc_tc", st);
+      if (p.kb_per_split <= 16) return launch_umma<16, true, false, 2, EPI_Z, 3>(tmX, tmYt, p, grid, "cols_acc_tc", st);
       return launch_umma<16, true, false, 2, EPI_Z, 5>(tmX, tmYt, p, grid, "cols_acc_tc", st);
     case 32: return launch_umma<32, true, false, 2, EPI_Z, 4>(tmX, tmYt, p, grid, "cols_acc_tc", st);
     default: return launch_umma<64, true, false, 2, EPI_Z, 3>(tmX, tmYt, p, grid, "cols_acc_tc", st);
